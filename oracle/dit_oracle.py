@@ -1,0 +1,249 @@
+"""CPU oracle for one DiT denoising step (TEST INFRASTRUCTURE, not a product path).
+
+A plain, slow NumPy fp64 statement of what the GPU library computes: a stack
+of adaLN-Zero DiT blocks applied to each request of a packed batch on its own.
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It shares no code with the CUDA path and imports neither it nor
+torch.
+
+What the paper fixes (Section 2 background and Section 2.1): a denoising step
+runs the transformer over a request's *full* latent token set, with attention
+giving every token global context; inference is stateless (Section 1); a
+request of H x W pixels has (H*W)/16^2 image tokens (Table 1, Section 6.1).
+The paper does not spell out the block, so the block below is the standard
+adaLN-Zero DiT block with the following readings (each is also listed in the
+design notes of the repository):
+
+  * sequential pre-LN block: attention branch, then MLP branch;
+  * cond -> modulation is Linear(SiLU(cond)) with bias, split into
+    (shift_a, scale_a, gate_a, shift_m, scale_m, gate_m), H each;
+  * LayerNorm over the H channels, biased variance, eps inside the root,
+    no learned affine;  modulate = LN(x) * (1 + scale) + shift;
+  * one weight set for image and text tokens; softmax scale 1/sqrt(d);
+    no mask inside a request, no other request visible; no positional term;
+  * GELU in its tanh form.
+
+Every function works on fp64 arrays.  Nothing is tiled, fused or reordered
+beyond taking query rows in slabs to bound memory (each softmax row is still
+the full definition over all keys of the request).
+
+Parity pins (tests/test_oracle_pins.py): hand-derived 2-token cases, softmax
+rows summing to one, zero gate => identity, row-permutation equivariance,
+packed (explicit block-diagonal mask) == each request alone, closed forms for
+LayerNorm / SiLU / GELU / modulation, Table 1 token counts for the packer.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Sequence, Tuple
+
+import numpy as np
+
+PATCH_PIXELS = 16
+
+Weights = Dict[str, np.ndarray]
+
+
+# --------------------------------------------------------------------------
+# request packing (integer, exact)
+# --------------------------------------------------------------------------
+def image_tokens(height: int, width: int) -> int:
+    """L = H*W / 16^2 (Section 6.1; Table 1 lists 256/1024/4096/16384)."""
+    if height <= 0 or width <= 0 or height % PATCH_PIXELS or width % PATCH_PIXELS:
+        raise ValueError("height and width must be positive multiples of 16")
+    return (height // PATCH_PIXELS) * (width // PATCH_PIXELS)
+
+
+def pack_requests(reqs: Sequence[Tuple[int, int, int]]):
+    """reqs: (height, width, n_text).  Returns token_lens, cu_seqlens, row_req, row_local.
+
+    Requests keep their input order; rows of request r occupy
+    [cu_seqlens[r], cu_seqlens[r+1]); inside a request image tokens come first.
+    """
+    lens = []
+    for (h, w, n_text) in reqs:
+        if n_text < 0:
+            raise ValueError("negative text token count")
+        lens.append(image_tokens(h, w) + n_text)
+    cu = [0]
+    for l in lens:
+        cu.append(cu[-1] + l)
+    row_req, row_local = [], []
+    for r, l in enumerate(lens):
+        for i in range(l):
+            row_req.append(r)
+            row_local.append(i)
+    return (np.array(lens, dtype=np.int32), np.array(cu, dtype=np.int32),
+            np.array(row_req, dtype=np.int32), np.array(row_local, dtype=np.int32))
+
+
+# --------------------------------------------------------------------------
+# block pieces
+# --------------------------------------------------------------------------
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def gelu_tanh(z: np.ndarray) -> np.ndarray:
+    return 0.5 * z * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (z + 0.044715 * z ** 3)))
+
+
+def layer_norm(x: np.ndarray, eps: float) -> np.ndarray:
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps)
+
+
+def adaln_modulation(cond: np.ndarray, w_ada: np.ndarray, b_ada: np.ndarray):
+    """cond [C] -> six vectors of H: shift_a, scale_a, gate_a, shift_m, scale_m, gate_m."""
+    m = silu(cond) @ w_ada + b_ada
+    return tuple(np.split(m, 6))
+
+
+def modulate(xhat: np.ndarray, shift: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    return xhat * (1.0 + scale) + shift
+
+
+def softmax_rows(s: np.ndarray) -> np.ndarray:
+    e = np.exp(s - s.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
+              rows: np.ndarray | None = None, slab: int = 2048) -> np.ndarray:
+    """Multi-head softmax attention over ONE request.  q,k,v: [L, H]; returns [len(rows), H].
+
+    Head j owns columns j*d .. (j+1)*d-1.  `rows` selects query rows (default all).
+    """
+    L, H = k.shape
+    d = H // n_heads
+    if rows is not None:
+        q = q[rows]
+    out = np.empty((q.shape[0], H), dtype=np.float64)
+    for j in range(n_heads):
+        cols = slice(j * d, (j + 1) * d)
+        kj, vj = k[:, cols], v[:, cols]
+        for r0 in range(0, q.shape[0], slab):
+            s = (q[r0:r0 + slab, cols] @ kj.T) / math.sqrt(d)
+            out[r0:r0 + slab, cols] = softmax_rows(s) @ vj
+    return out
+
+
+def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps: float,
+                  rows: np.ndarray | None = None, taps: dict | None = None) -> np.ndarray:
+    """One adaLN-Zero DiT block on one request.  x [L, H], cond [C] -> [L, H].
+
+    With `rows`, only those output rows are produced (keys and values still
+    come from every row of the request); used to sample outputs of long
+    sequences.  `taps`, if given, receives the intermediates h1, qkv, a, x_mid,
+    h2, u for per-kernel comparisons.
+    """
+    H = x.shape[1]
+    shift_a, scale_a, gate_a, shift_m, scale_m, gate_m = adaln_modulation(cond, w["w_ada"], w["b_ada"])
+    h = modulate(layer_norm(x, eps), shift_a, scale_a)
+    qkv = h @ w["w_qkv"] + w["b_qkv"]
+    q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+    a = attention(q, k, v, n_heads, rows)
+    xr = x if rows is None else x[rows]
+    x_mid = xr + gate_a * (a @ w["w_o"] + w["b_o"])
+    h2 = modulate(layer_norm(x_mid, eps), shift_m, scale_m)
+    u = gelu_tanh(h2 @ w["w_fc1"] + w["b_fc1"])
+    y = x_mid + gate_m * (u @ w["w_fc2"] + w["b_fc2"])
+    if taps is not None:
+        taps.update(h1=h, qkv=qkv, a=a, x_mid=x_mid, h2=h2, u=u)
+    return y
+
+
+def stack_forward_alone(x: np.ndarray, cond: np.ndarray, blocks: Sequence[Weights],
+                        n_heads: int, eps: float) -> np.ndarray:
+    """A stack of blocks on one request run by itself."""
+    for w in blocks:
+        x = block_forward(x, cond, w, n_heads, eps)
+    return x
+
+
+def step_forward(packed: np.ndarray, token_lens: Sequence[int], cond: np.ndarray,
+                 blocks: Sequence[Weights], n_heads: int, eps: float) -> np.ndarray:
+    """One denoising step over a packed batch: each request through the stack on its own."""
+    out = np.empty_like(packed)
+    p = 0
+    for r, l in enumerate(token_lens):
+        out[p:p + l] = stack_forward_alone(packed[p:p + l], cond[r], blocks, n_heads, eps)
+        p += l
+    return out
+
+
+def step_forward_masked(packed: np.ndarray, token_lens: Sequence[int], cond: np.ndarray,
+                        blocks: Sequence[Weights], n_heads: int, eps: float) -> np.ndarray:
+    """Second, independent statement of the packed step (small cases only).
+
+    Works on the whole [T, H] batch at once: per-row modulation vectors looked
+    up through row -> request, and ONE T x T score matrix per head with an
+    explicit block-diagonal mask (-inf outside a row's own request).
+    """
+    T, H = packed.shape
+    d = H // n_heads
+    row_req = np.repeat(np.arange(len(token_lens)), token_lens)
+    same = row_req[:, None] == row_req[None, :]
+    x = packed.copy()
+    for w in blocks:
+        mod = np.stack([silu(c) @ w["w_ada"] + w["b_ada"] for c in cond])[row_req]   # [T, 6H]
+        sh_a, sc_a, g_a, sh_m, sc_m, g_m = (mod[:, i * H:(i + 1) * H] for i in range(6))
+        h = layer_norm(x, eps) * (1.0 + sc_a) + sh_a
+        qkv = h @ w["w_qkv"] + w["b_qkv"]
+        a = np.empty_like(x)
+        for j in range(n_heads):
+            q = qkv[:, j * d:(j + 1) * d]
+            k = qkv[:, H + j * d:H + (j + 1) * d]
+            v = qkv[:, 2 * H + j * d:2 * H + (j + 1) * d]
+            s = np.where(same, (q @ k.T) / math.sqrt(d), -np.inf)
+            a[:, j * d:(j + 1) * d] = softmax_rows(s) @ v
+        x = x + g_a * (a @ w["w_o"] + w["b_o"])
+        h = layer_norm(x, eps) * (1.0 + sc_m) + sh_m
+        x = x + g_m * (gelu_tanh(h @ w["w_fc1"] + w["b_fc1"]) @ w["w_fc2"] + w["b_fc2"])
+    return x
+
+
+def block_forward_scalar(x: Sequence[Sequence[float]], cond: Sequence[float], w: Weights,
+                         n_heads: int, eps: float) -> List[List[float]]:
+    """Third statement, pure-Python scalar loops (tiny cases only): no NumPy arithmetic."""
+    L, H = len(x), len(x[0])
+    C = len(cond)
+    d = H // n_heads
+    W = {k: np.asarray(v).tolist() for k, v in w.items()}
+    sc = [c / (1.0 + math.exp(-c)) for c in cond]
+    m = [sum(sc[i] * W["w_ada"][i][o] for i in range(C)) + W["b_ada"][o] for o in range(6 * H)]
+    part = [m[i * H:(i + 1) * H] for i in range(6)]
+
+    def ln_mod(row, shift, scale):
+        mu = sum(row) / H
+        var = sum((t - mu) ** 2 for t in row) / H
+        return [(row[c] - mu) / math.sqrt(var + eps) * (1.0 + scale[c]) + shift[c] for c in range(H)]
+
+    def linear(row, wname, bname):
+        wm, b = W[wname], W[bname]
+        return [sum(row[i] * wm[i][o] for i in range(len(row))) + b[o] for o in range(len(b))]
+
+    h = [ln_mod(r, part[0], part[1]) for r in x]
+    qkv = [linear(r, "w_qkv", "b_qkv") for r in h]
+    a = [[0.0] * H for _ in range(L)]
+    for j in range(n_heads):
+        for i in range(L):
+            s = [sum(qkv[i][j * d + c] * qkv[t][H + j * d + c] for c in range(d)) / math.sqrt(d) for t in range(L)]
+            e = [math.exp(v) for v in s]
+            z = sum(e)
+            for c in range(d):
+                a[i][j * d + c] = sum(e[t] / z * qkv[t][2 * H + j * d + c] for t in range(L))
+    proj = [linear(r, "w_o", "b_o") for r in a]
+    xm = [[x[i][c] + part[2][c] * proj[i][c] for c in range(H)] for i in range(L)]
+    h2 = [ln_mod(r, part[3], part[4]) for r in xm]
+    pre = [linear(r, "w_fc1", "b_fc1") for r in h2]
+    u = [[0.5 * z * (1.0 + math.tanh(math.sqrt(2.0 / math.pi) * (z + 0.044715 * z * z * z))) for z in r] for r in pre]
+    f2 = [linear(r, "w_fc2", "b_fc2") for r in u]
+    return [[xm[i][c] + part[5][c] * f2[i][c] for c in range(H)] for i in range(L)]
+
+
+def error_metric(got: np.ndarray, ref: np.ndarray) -> float:
+    """max|got - ref| / rms(ref) over one request's outputs."""
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.abs(np.asarray(got, dtype=np.float64) - ref).max() / math.sqrt(np.mean(ref ** 2)))
