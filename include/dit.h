@@ -1,0 +1,162 @@
+/*
+ * libdit — one denoising step of a Diffusion Transformer on one B200 (sm_100a).
+ *
+ * The paper's serving system dispatches, per scheduling round, "diffusion steps" of requests to
+ * GPU workers (Section 4, request lifecycle; Section 3 problem formulation: a request has a
+ * resolution and S_i strictly dependent steps, one running at a time).  This library is the
+ * single-GPU step those schedules dispatch: a stack of adaLN-Zero DiT blocks run over a batch of
+ * requests at mixed image resolutions, packed into one variable-length batch with block-diagonal
+ * attention per request (the mechanism behind the paper's batching of small-resolution steps,
+ * Section 5 "selective continuous batching", generalised to mixed lengths).
+ *
+ * Conventions
+ *   - C ABI, no exceptions, nothing aborts or prints.  Every call returns a dit_status; on error
+ *     no kernel has been launched by that call unless stated otherwise.
+ *   - "device" pointers are CUDA device memory of the current device, "HOST" pointers are host
+ *     memory.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Tokens, cond and weights cross the boundary as bf16; `out` is fp32.  Inside, GEMM operands
+ *     are fp16 (bf16 weights ~N(0,0.02) convert exactly), accumulation, the residual stream and the
+ *     modulation vectors are fp32.
+ *   - The caller owns every buffer, including the workspace; the context owns only what it carves
+ *     from the workspace.  No entry point below allocates device memory.
+ *   - A context is not thread-safe; calls on one context must be issued serially (they may be
+ *     asynchronous on one stream).
+ *
+ * The block (per request r, tokens x [L_r, H], cond c [C]); the paper runs such blocks through
+ * PyTorch and does not restate them, so this is the standard adaLN-Zero form:
+ *   m = W_ada^T SiLU(c) + b_ada, split as (shift_a, scale_a, gate_a, shift_m, scale_m, gate_m)
+ *   h = LN(x) * (1 + scale_a) + shift_a            LN over H, biased variance, eps, no affine
+ *   [Q|K|V] = h W_qkv + b_qkv                       head j = columns j*d..(j+1)*d-1 of each third
+ *   a = concat_j softmax(Q_j K_j^T / sqrt(d)) V_j   over the L_r tokens of this request only
+ *   x = x + gate_a * (a W_o + b_o)
+ *   h = LN(x) * (1 + scale_m) + shift_m
+ *   x = x + gate_m * (gelu_tanh(h W_1 + b_1) W_2 + b_2)
+ */
+#ifndef DIT_H_
+#define DIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DIT_MAX_REQUESTS 64 /* upper bound on dit_config.max_requests */
+
+typedef struct dit_ctx dit_ctx; /* opaque */
+
+typedef enum {
+  DIT_OK = 0,
+  DIT_ERR_INVALID_ARG = 1,      /* NULL pointer, negative count, bad index */
+  DIT_ERR_SHAPE = 2,            /* dimensions the kernels do not support, lengths that do not add up */
+  DIT_ERR_CAPACITY = 3,         /* more tokens / requests / blocks than the context was sized for */
+  DIT_ERR_NOT_LOADED = 4,       /* a block in [0, n_blocks) has no weights yet */
+  DIT_ERR_UNSUPPORTED_ARCH = 5, /* the current device is not compute capability 10.x */
+  DIT_ERR_CUDA = 6,             /* a CUDA runtime/driver call failed; see dit_last_error */
+  DIT_ERR_TIMEOUT = 7,          /* a kernel gave up on a bounded wait (device status word) */
+  DIT_ERR_INTERNAL = 8
+} dit_status;
+
+typedef struct {
+  int32_t hidden;           /* H; multiple of 64, <= 8192 */
+  int32_t n_heads;          /* nh; H = nh * head_dim */
+  int32_t head_dim;         /* d; 64 or 128 */
+  int32_t mlp_hidden;       /* F; multiple of 64 */
+  int32_t cond_dim;         /* C; multiple of 8 */
+  int32_t max_blocks;       /* weight slots carved from the workspace */
+  int32_t max_total_tokens; /* capacity T_max of one packed batch */
+  int32_t max_requests;     /* capacity R_max, <= DIT_MAX_REQUESTS */
+  float ln_eps;             /* LayerNorm epsilon (1e-6 in every benchmark configuration) */
+  uint32_t flags;           /* reserved, must be 0 */
+} dit_config;
+
+/* One request of the paper's problem statement (Section 3): an image resolution, a position in
+ * its denoising schedule and the diffusion time of this step.  Image tokens = (height/16) *
+ * (width/16) (Section 6.1: L = H*W/16^2; Table 1: 256/1024/4096/16384 for 256^2..2048^2). */
+typedef struct {
+  int32_t height, width;  /* pixels, positive multiples of 16 */
+  int32_t n_text_tokens;  /* >= 0; appended after the image tokens of the request */
+  float timestep;         /* t of this step; carried for the caller, the cond vector already encodes it */
+  int32_t step_index;     /* which of the request's S_i steps this is; carried for the caller */
+} dit_request;
+
+/* Device pointers, bf16, row-major [in, out] (y = x W + b).  A NULL bias means zero.
+ *   w_ada [C, 6H]  b_ada [6H]   chunk order: shift_a, scale_a, gate_a, shift_m, scale_m, gate_m
+ *   w_qkv [H, 3H]  b_qkv [3H]   columns: Q | K | V
+ *   w_o   [H, H]   b_o   [H]
+ *   w_fc1 [H, F]   b_fc1 [F]
+ *   w_fc2 [F, H]   b_fc2 [H] */
+typedef struct {
+  const void *w_ada, *b_ada, *w_qkv, *b_qkv, *w_o, *b_o, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+} dit_block_weights;
+
+/* Bytes of device workspace a context of this configuration needs (0 if the configuration is
+ * invalid).  Covers converted weights for max_blocks blocks, the fp32 residual stream, the
+ * intermediate activations, the modulation vectors and staging for dit_step_forward_host. */
+size_t dit_workspace_bytes(const dit_config *cfg);
+
+/* Creates a context on the current device.  `workspace` is device memory, 1024-byte aligned, at
+ * least dit_workspace_bytes(cfg) long; it must outlive the context.  Fails with
+ * DIT_ERR_UNSUPPORTED_ARCH on anything but sm_100 (there is no fallback path). */
+dit_status dit_ctx_create(const dit_config *cfg, void *workspace, size_t workspace_bytes, dit_ctx **out);
+dit_status dit_ctx_destroy(dit_ctx *ctx);
+
+/* Copies block `block_idx`'s ten tensors into the context (weights are re-laid out as fp16
+ * [out, in] for the tensor-core kernels, biases widened to fp32).  Asynchronous on `stream`; the
+ * caller's tensors may be freed once the stream has passed this point. */
+dit_status dit_load_block_weights(dit_ctx *ctx, int32_t block_idx, const dit_block_weights *w, void *stream);
+
+/* Packer, host only, integer only (Section 6.1 token rule; requests keep their input order; inside
+ * a request image tokens come first, then text tokens).  All arrays are HOST memory owned by the
+ * caller: token_lens [n], cu_seqlens [n+1], row_req / row_local [sum of lens] (either may be NULL).
+ * total_tokens receives the sum.  n == 0 is valid.  DIT_ERR_SHAPE for a resolution that is not a
+ * positive multiple of 16 or a negative text length. */
+dit_status dit_pack_requests(const dit_request *reqs, int32_t n, int32_t *token_lens, int32_t *cu_seqlens,
+                             int32_t *row_req, int32_t *row_local, int32_t *total_tokens);
+
+/* Gathers n per-request device buffers [L_r, H] bf16 (HOST array of device pointers) into one packed
+ * device buffer [sum L_r, H] bf16 in request order.  Asynchronous on `stream`. */
+dit_status dit_pack_tokens(dit_ctx *ctx, const void *const *per_request_tokens, const int32_t *token_lens,
+                           int32_t n, void *packed_tokens, void *stream);
+
+/* One denoising step: blocks 0..n_blocks-1 over the packed batch.
+ *   packed_tokens           device [T, H] bf16, T = sum of lens; request r owns rows
+ *                           [cu[r], cu[r+1]) in input order
+ *   per_request_token_lens  HOST [n_requests] int32, each >= 1; read before the call returns
+ *   per_request_cond        device [n_requests, C] bf16; row r conditions request r
+ *   out                     device [T, H] fp32
+ * Asynchronous on `stream`; never allocates.  n_requests == 0 is a no-op.  Errors are detected on
+ * the host before any launch (DIT_ERR_CAPACITY, DIT_ERR_NOT_LOADED, DIT_ERR_INVALID_ARG). */
+dit_status dit_step_forward(dit_ctx *ctx, const void *packed_tokens, const int32_t *per_request_token_lens,
+                            int32_t n_requests, const void *per_request_cond, int32_t n_blocks, float *out,
+                            void *stream);
+
+/* Same step with HOST buffers: copies tokens and cond to the device, runs the step, copies `out`
+ * back, all on `stream`, and returns after the stream has drained (out is valid on return).
+ * Pinned host memory makes the copies asynchronous with respect to other streams. */
+dit_status dit_step_forward_host(dit_ctx *ctx, const void *host_packed_tokens,
+                                 const int32_t *per_request_token_lens, int32_t n_requests,
+                                 const void *host_cond, int32_t n_blocks, float *host_out, void *stream);
+
+/* Reads (with a device synchronisation) the device status word that kernels set when a bounded wait
+ * runs out; returns DIT_OK or DIT_ERR_TIMEOUT and clears the word. */
+dit_status dit_ctx_poll_status(dit_ctx *ctx);
+
+/* Test hook: device pointers to the context's intermediates of the LAST block run by the last
+ * step (h = second LayerNorm+modulate output, qkv, a = attention output, u = GELU output are fp16;
+ * mod [R, n_blocks, 6H] and stream [T, H] are fp32).  Valid until the next call on the context. */
+typedef enum { DIT_TAP_H = 0, DIT_TAP_QKV = 1, DIT_TAP_ATTN = 2, DIT_TAP_U = 3, DIT_TAP_MOD = 4, DIT_TAP_STREAM = 5 } dit_tap;
+dit_status dit_debug_tap(dit_ctx *ctx, dit_tap which, const void **ptr, int64_t *rows, int64_t *cols,
+                         int32_t *elem_bytes);
+
+/* Number of kernel launches issued by the last dit_step_forward on this context. */
+int64_t dit_last_launch_count(const dit_ctx *ctx);
+
+const char *dit_status_string(dit_status s);
+const char *dit_last_error(const dit_ctx *ctx); /* detail of the last failure on this context ("" if none) */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIT_H_ */

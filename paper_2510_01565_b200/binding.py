@@ -1,0 +1,261 @@
+"""ctypes binding of libdit.so: argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels; torch is used
+here for device memory and streams.  Loading fails loudly when the library has
+not been built (there is no CPU or eager fallback).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdit.so")
+
+DIT_OK = 0
+STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
+                "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
+TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
+
+EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
+           "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_host",
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
+
+
+class DitConfig(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("mlp_hidden", C.c_int32),
+                ("cond_dim", C.c_int32), ("max_blocks", C.c_int32), ("max_total_tokens", C.c_int32),
+                ("max_requests", C.c_int32), ("ln_eps", C.c_float), ("flags", C.c_uint32)]
+
+
+class DitRequest(C.Structure):
+    _fields_ = [("height", C.c_int32), ("width", C.c_int32), ("n_text_tokens", C.c_int32),
+                ("timestep", C.c_float), ("step_index", C.c_int32)]
+
+
+class DitBlockWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o",
+                                          "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
+
+
+class DitError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{name}: {detail}" if detail else name)
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libdit.so and declares the signatures of include/dit.h."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_01565_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    lib.dit_workspace_bytes.restype = C.c_size_t
+    lib.dit_workspace_bytes.argtypes = [C.POINTER(DitConfig)]
+    lib.dit_ctx_create.restype = C.c_int
+    lib.dit_ctx_create.argtypes = [C.POINTER(DitConfig), vp, C.c_size_t, C.POINTER(vp)]
+    lib.dit_ctx_destroy.restype = C.c_int
+    lib.dit_ctx_destroy.argtypes = [vp]
+    lib.dit_load_block_weights.restype = C.c_int
+    lib.dit_load_block_weights.argtypes = [vp, i32, C.POINTER(DitBlockWeights), vp]
+    lib.dit_pack_requests.restype = C.c_int
+    lib.dit_pack_requests.argtypes = [C.POINTER(DitRequest), i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32),
+                                      C.POINTER(i32), C.POINTER(i32)]
+    lib.dit_pack_tokens.restype = C.c_int
+    lib.dit_pack_tokens.argtypes = [vp, C.POINTER(vp), C.POINTER(i32), i32, vp, vp]
+    lib.dit_step_forward.restype = C.c_int
+    lib.dit_step_forward.argtypes = [vp, vp, C.POINTER(i32), i32, vp, i32, vp, vp]
+    lib.dit_step_forward_host.restype = C.c_int
+    lib.dit_step_forward_host.argtypes = [vp, vp, C.POINTER(i32), i32, vp, i32, vp, vp]
+    lib.dit_ctx_poll_status.restype = C.c_int
+    lib.dit_ctx_poll_status.argtypes = [vp]
+    lib.dit_debug_tap.restype = C.c_int
+    lib.dit_debug_tap.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+    lib.dit_last_launch_count.restype = i64
+    lib.dit_last_launch_count.argtypes = [vp]
+    lib.dit_status_string.restype = C.c_char_p
+    lib.dit_status_string.argtypes = [C.c_int]
+    lib.dit_last_error.restype = C.c_char_p
+    lib.dit_last_error.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+def dit_pack_requests(reqs: Sequence[Sequence]) -> Dict[str, np.ndarray]:
+    """reqs: (height, width, n_text[, timestep, step_index]).  Host-only; returns int32 arrays."""
+    lib = load_library()
+    n = len(reqs)
+    arr = (DitRequest * max(n, 1))()
+    for i, r in enumerate(reqs):
+        arr[i] = DitRequest(int(r[0]), int(r[1]), int(r[2]), float(r[3]) if len(r) > 3 else 0.0,
+                            int(r[4]) if len(r) > 4 else 0)
+    lens = np.zeros(max(n, 1), dtype=np.int32)
+    cu = np.zeros(n + 1, dtype=np.int32)
+    total = C.c_int32(0)
+    ip = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    st = lib.dit_pack_requests(arr, n, ip(lens), ip(cu), None, None, C.byref(total))
+    if st != DIT_OK:
+        raise DitError(st)
+    row_req = np.zeros(max(total.value, 1), dtype=np.int32)
+    row_local = np.zeros(max(total.value, 1), dtype=np.int32)
+    st = lib.dit_pack_requests(arr, n, ip(lens), ip(cu), ip(row_req), ip(row_local), C.byref(total))
+    if st != DIT_OK:
+        raise DitError(st)
+    return {"token_lens": lens[:n], "cu_seqlens": cu, "row_req": row_req[:total.value],
+            "row_local": row_local[:total.value], "total_tokens": total.value}
+
+
+class DitContext:
+    """Owns a workspace tensor and a dit_ctx on the current CUDA device."""
+
+    def __init__(self, hidden: int, n_heads: int, head_dim: int, mlp_hidden: int, cond_dim: int,
+                 max_blocks: int, max_total_tokens: int, max_requests: int = 8, ln_eps: float = 1e-6):
+        import torch
+        self.torch = torch
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("libdit needs a CUDA device (sm_100); there is no CPU path")
+        self.cfg = DitConfig(hidden, n_heads, head_dim, mlp_hidden, cond_dim, max_blocks, max_total_tokens,
+                             max_requests, ln_eps, 0)
+        nbytes = self.lib.dit_workspace_bytes(C.byref(self.cfg))
+        if nbytes == 0:
+            raise DitError(2, "configuration rejected by dit_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
+        base = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+        self.workspace_bytes = nbytes
+        handle = C.c_void_p()
+        st = self.lib.dit_ctx_create(C.byref(self.cfg), C.c_void_p(base), nbytes, C.byref(handle))
+        if st != DIT_OK:
+            raise DitError(st, "dit_ctx_create")
+        self.handle = handle
+        self.hidden, self.cond_dim, self.mlp_hidden = hidden, cond_dim, mlp_hidden
+
+    # ------------------------------------------------------------------ helpers
+    def _check(self, st: int):
+        if st != DIT_OK:
+            raise DitError(st, self.lib.dit_last_error(self.handle).decode())
+
+    def _stream(self, stream=None) -> C.c_void_p:
+        s = self.torch.cuda.current_stream() if stream is None else stream
+        return C.c_void_p(s.cuda_stream)
+
+    @staticmethod
+    def _lens(lens) -> np.ndarray:
+        return np.ascontiguousarray(np.asarray(lens, dtype=np.int32))
+
+    def close(self):
+        if getattr(self, "handle", None) is not None:
+            self.torch.cuda.synchronize()
+            self.lib.dit_ctx_destroy(self.handle)
+            self.handle = None
+            self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ C-ABI calls
+    def dit_load_block_weights(self, block_idx: int, weights: Dict[str, "object"], stream=None):
+        """weights: name -> CUDA bf16 tensor, [in, out] row-major; biases may be None."""
+        w = DitBlockWeights()
+        keep = []
+        for name, _ in DitBlockWeights._fields_:
+            t = weights.get(name)
+            if t is None:
+                setattr(w, name, None)
+                continue
+            assert t.is_cuda and t.dtype == self.torch.bfloat16 and t.is_contiguous(), name
+            keep.append(t)
+            setattr(w, name, t.data_ptr())
+        self._check(self.lib.dit_load_block_weights(self.handle, block_idx, C.byref(w), self._stream(stream)))
+
+    def dit_pack_tokens(self, per_request_tokens: List["object"], stream=None):
+        torch = self.torch
+        n = len(per_request_tokens)
+        lens = self._lens([t.shape[0] for t in per_request_tokens])
+        for t in per_request_tokens:
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape[1] == self.hidden
+        packed = torch.empty((int(lens.sum()), self.hidden), dtype=torch.bfloat16, device="cuda")
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in per_request_tokens])
+        self._check(self.lib.dit_pack_tokens(self.handle, ptrs, lens.ctypes.data_as(C.POINTER(C.c_int32)), n,
+                                             C.c_void_p(packed.data_ptr()), self._stream(stream)))
+        return packed
+
+    def dit_step_forward(self, packed_tokens, token_lens, cond, n_blocks: int, out=None, stream=None):
+        """packed_tokens [T,H] bf16 cuda, cond [R,C] bf16 cuda -> out [T,H] fp32 cuda (asynchronous)."""
+        torch = self.torch
+        lens = self._lens(token_lens)
+        assert packed_tokens.is_cuda and packed_tokens.dtype == torch.bfloat16 and packed_tokens.is_contiguous()
+        assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous()
+        assert packed_tokens.shape == (int(lens.sum()), self.hidden) and cond.shape == (len(lens), self.cond_dim)
+        if out is None:
+            out = torch.empty(packed_tokens.shape, dtype=torch.float32, device="cuda")
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.shape == packed_tokens.shape
+        self._check(self.lib.dit_step_forward(self.handle, C.c_void_p(packed_tokens.data_ptr()),
+                                              lens.ctypes.data_as(C.POINTER(C.c_int32)), len(lens),
+                                              C.c_void_p(cond.data_ptr()), n_blocks, C.c_void_p(out.data_ptr()),
+                                              self._stream(stream)))
+        return out
+
+    def dit_step_forward_host(self, host_tokens, token_lens, host_cond, n_blocks: int, host_out, stream=None):
+        """Host (ideally pinned) torch tensors in and out; returns after `out` is valid."""
+        lens = self._lens(token_lens)
+        assert not host_tokens.is_cuda and not host_cond.is_cuda and not host_out.is_cuda
+        assert host_tokens.is_contiguous() and host_cond.is_contiguous() and host_out.is_contiguous()
+        assert host_tokens.shape == (int(lens.sum()), self.hidden) and host_out.shape == host_tokens.shape
+        self._check(self.lib.dit_step_forward_host(self.handle, C.c_void_p(host_tokens.data_ptr()),
+                                                   lens.ctypes.data_as(C.POINTER(C.c_int32)), len(lens),
+                                                   C.c_void_p(host_cond.data_ptr()), n_blocks,
+                                                   C.c_void_p(host_out.data_ptr()), self._stream(stream)))
+        return host_out
+
+    def dit_ctx_poll_status(self):
+        self._check(self.lib.dit_ctx_poll_status(self.handle))
+
+    def dit_last_launch_count(self) -> int:
+        return int(self.lib.dit_last_launch_count(self.handle))
+
+    def dit_debug_tap(self, which: str):
+        """Copy of an internal buffer of the last step as a torch tensor (fp16 or fp32)."""
+        torch = self.torch
+        ptr, rows, cols, eb = C.c_void_p(), C.c_int64(), C.c_int64(), C.c_int32()
+        self._check(self.lib.dit_debug_tap(self.handle, TAPS[which], C.byref(ptr), C.byref(rows), C.byref(cols), C.byref(eb)))
+        dtype = torch.float16 if eb.value == 2 else torch.float32
+        base = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+        off = ptr.value - base
+        torch.cuda.synchronize()
+        flat = self.workspace[(base - self.workspace.data_ptr()) + off:(base - self.workspace.data_ptr()) + off + rows.value * cols.value * eb.value]
+        return flat.view(dtype).view(rows.value, cols.value).clone()
+
+
+def context_for(dims, max_blocks: int, max_total_tokens: int, max_requests: int = 8) -> DitContext:
+    return DitContext(dims.hidden, dims.n_heads, dims.head_dim, dims.mlp_hidden, dims.cond_dim,
+                      max_blocks, max_total_tokens, max_requests, dims.ln_eps)
+
+
+def upload_weights(ctx: DitContext, blocks) -> None:
+    """blocks: list of dicts name -> numpy uint16 (bf16 bits).  Copies to the GPU and loads them."""
+    import torch
+    for b, w in enumerate(blocks):
+        dev = {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in w.items()}
+        ctx.dit_load_block_weights(b, dev)
+        torch.cuda.synchronize()
+        del dev
+
+
+def bits_to_cuda_bf16(bits: np.ndarray):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)

@@ -1,0 +1,36 @@
+// Types shared by the kernels of libdit.
+#pragma once
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dit.h"
+
+namespace dit {
+
+// Packed-batch description, passed by value as a kernel parameter (no device-side plan buffer):
+// cu[r] .. cu[r+1] are the packed rows of request r.  `order` lists requests longest first (used by
+// the attention grid so that long requests start early).
+struct SeqInfo {
+  int n;
+  int total;
+  int cu[DIT_MAX_REQUESTS + 1];
+  int order[DIT_MAX_REQUESTS];
+};
+
+// Device status word values (written by a kernel whose bounded wait ran out).
+enum : int { kStatusOk = 0, kStatusGemmTimeout = 1, kStatusAttnTimeout = 2 };
+
+// Request that owns packed row `row` (binary search over at most 64 entries).
+__device__ __forceinline__ int find_request(const SeqInfo& s, int row) {
+  int lo = 0, hi = s.n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (s.cu[mid] <= row) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+}  // namespace dit

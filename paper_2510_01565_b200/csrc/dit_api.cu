@@ -1,0 +1,504 @@
+// libdit: C ABI, context, host-side planning and kernel launches.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "gemm.cuh"
+
+using namespace dit;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t kAlign = 1024;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Offsets (bytes) inside one block's weight slot.
+struct BlockLayout {
+  size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, bytes;
+};
+// Offsets (bytes) inside the workspace.
+struct Layout {
+  BlockLayout blk;
+  size_t weights, stream, h, qkv, a, u, mod, status, stage_tokens, stage_cond, stage_out, bytes;
+};
+
+bool config_ok(const dit_config* c) {
+  if (!c) return false;
+  if (c->hidden < 64 || c->hidden % 64 || c->hidden > 4096) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_heads < 1 || static_cast<long long>(c->n_heads) * c->head_dim != c->hidden) return false;
+  if (c->mlp_hidden < 64 || c->mlp_hidden % 64) return false;
+  if (c->cond_dim < 1 || c->cond_dim > 4096) return false;
+  if (c->max_blocks < 1 || c->max_total_tokens < 1) return false;
+  if (c->max_requests < 1 || c->max_requests > DIT_MAX_REQUESTS) return false;
+  if (!(c->ln_eps >= 0.f) || c->flags != 0) return false;
+  return true;
+}
+
+Layout make_layout(const dit_config& c) {
+  const size_t H = c.hidden, F = c.mlp_hidden, C = c.cond_dim, T = c.max_total_tokens, R = c.max_requests;
+  Layout L{};
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  L.blk.w_ada = take(C * 6 * H * 2);
+  L.blk.b_ada = take(6 * H * 4);
+  L.blk.w_qkv = take(3 * H * H * 2);
+  L.blk.b_qkv = take(3 * H * 4);
+  L.blk.w_o = take(H * H * 2);
+  L.blk.b_o = take(H * 4);
+  L.blk.w_fc1 = take(F * H * 2);
+  L.blk.b_fc1 = take(F * 4);
+  L.blk.w_fc2 = take(H * F * 2);
+  L.blk.b_fc2 = take(H * 4);
+  L.blk.bytes = o;
+  o = 0;
+  L.weights = take(L.blk.bytes * c.max_blocks);
+  L.stream = take(T * H * 4);
+  L.h = take(T * H * 2);
+  L.qkv = take(T * 3 * H * 2);
+  L.a = take(T * H * 2);
+  L.u = take(T * F * 2);
+  L.mod = take(R * c.max_blocks * 6 * H * 4);
+  L.status = take(256);
+  L.stage_tokens = take(T * H * 2);
+  L.stage_cond = take(R * C * 2);
+  L.stage_out = take(T * H * 4);
+  L.bytes = o;
+  return L;
+}
+
+struct BlockState {
+  bool loaded = false;
+  CUtensorMap tm_qkv, tm_o, tm_fc1, tm_fc2;
+};
+
+}  // namespace
+
+struct dit_ctx {
+  dit_config cfg;
+  Layout lay;
+  uint8_t* ws;
+  EncodeTiledFn encode;
+  int num_sms;
+  BlockState* blocks;
+  int64_t last_launches;
+  int last_T, last_R, last_nb;
+  char err[256];
+
+  template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  uint8_t* block_base(int b) const { return ws + lay.weights + lay.blk.bytes * static_cast<size_t>(b); }
+};
+
+namespace {
+
+dit_status fail(dit_ctx* ctx, dit_status s, const char* fmt, const char* detail = "") {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), fmt, detail);
+  return s;
+}
+
+#define DIT_CUDA_TRY(ctx, expr)                                                        \
+  do {                                                                                 \
+    cudaError_t e_ = (expr);                                                           \
+    if (e_ != cudaSuccess) return fail(ctx, DIT_ERR_CUDA, #expr ": %s", cudaGetErrorString(e_)); \
+  } while (0)
+
+// 2-D fp16 tensor map: `inner` contiguous elements per row, `rows` rows, box 64 x box_rows, 128-byte swizzle,
+// out-of-bounds elements read as zero.
+bool make_map(const dit_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
+  s->n = n;
+  s->cu[0] = 0;
+  for (int r = 0; r < n; ++r) {
+    if (lens[r] < 1) return false;
+    s->cu[r + 1] = s->cu[r] + lens[r];
+    s->order[r] = r;
+  }
+  s->total = s->cu[n];
+  std::stable_sort(s->order, s->order + n, [&](int a, int b) { return lens[a] > lens[b]; });
+  return true;
+}
+
+template <int EPI>
+cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
+                        const SeqInfo& seq, cudaStream_t st) {
+  const int tiles = ((p.M + gemm_cfg::BM - 1) / gemm_cfg::BM) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
+  const int grid = std::min(tiles, ctx->num_sms);
+  gemm_tcgen05_kernel<EPI><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, p, seq);
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, const SeqInfo& seq, cudaStream_t st) {
+  int qtiles = 0;
+  for (int r = 0; r < seq.n; ++r) qtiles += (seq.cu[r + 1] - seq.cu[r] + 127) / 128;
+  attention_tcgen05_kernel<D><<<qtiles * p.n_heads, AttnCfg<D>::THREADS, AttnCfg<D>::SMEM_BYTES, st>>>(tmQKV, p, seq);
+  return cudaGetLastError();
+}
+
+size_t mod_smem_bytes(int C) { return (static_cast<size_t>(kModReqGroup) * C + 8 * kModReqGroup * kModCols) * sizeof(float); }
+
+dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
+                     float* out, cudaStream_t st) {
+  const dit_config& c = ctx->cfg;
+  SeqInfo seq{};
+  if (!build_seq(lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
+  const int T = seq.total, H = c.hidden, F = c.mlp_hidden;
+  if (T > c.max_total_tokens) return fail(ctx, DIT_ERR_CAPACITY, "packed batch exceeds max_total_tokens");
+  for (int b = 0; b < n_blocks; ++b)
+    if (!ctx->blocks[b].loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "a block in [0, n_blocks) has no weights");
+
+  float* stream = ctx->at<float>(ctx->lay.stream);
+  __half* h = ctx->at<__half>(ctx->lay.h);
+  __half* qkv = ctx->at<__half>(ctx->lay.qkv);
+  __half* a = ctx->at<__half>(ctx->lay.a);
+  __half* u = ctx->at<__half>(ctx->lay.u);
+  float* mod = ctx->at<float>(ctx->lay.mod);
+  int* status = ctx->at<int>(ctx->lay.status);
+
+  CUtensorMap tm_h, tm_a, tm_u, tm_qkv;
+  if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM) || !make_map(ctx, &tm_a, a, H, T, gemm_cfg::BM) ||
+      !make_map(ctx, &tm_u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &tm_qkv, qkv, 3 * H, T, 128))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+
+  int64_t launches = 0;
+  const long long req_stride = static_cast<long long>(n_blocks) * 6 * H;
+
+  {  // adaLN modulation vectors of every block
+    ModParams mp{};
+    mp.cond = static_cast<const __nv_bfloat16*>(cond);
+    mp.w_ada0 = reinterpret_cast<const __nv_bfloat16*>(ctx->block_base(0) + ctx->lay.blk.w_ada);
+    mp.b_ada0 = reinterpret_cast<const float*>(ctx->block_base(0) + ctx->lay.blk.b_ada);
+    mp.w_block_stride = static_cast<long long>(ctx->lay.blk.bytes / 2);
+    mp.b_block_stride = static_cast<long long>(ctx->lay.blk.bytes / 4);
+    mp.mod = mod; mp.R = n; mp.C = c.cond_dim; mp.N6 = 6 * H; mp.NB = n_blocks;
+    const int grid = n_blocks * ((6 * H + kModCols - 1) / kModCols);
+    modulation_kernel<<<grid, kModThreads, mod_smem_bytes(c.cond_dim), st>>>(mp);
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    ++launches;
+  }
+
+  const int ln_grid = (T + kLnWarps - 1) / kLnWarps;
+  for (int b = 0; b < n_blocks; ++b) {
+    const BlockState& bs = ctx->blocks[b];
+    const uint8_t* wb = ctx->block_base(b);
+    const float* modb = mod + static_cast<size_t>(b) * 6 * H;   // request 0; request r at + r * req_stride
+    // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
+    if (b == 0)
+      ln_modulate_kernel<true><<<ln_grid, kLnWarps * 32, 0, st>>>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
+    else
+      ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    // QKV projection
+    GemmParams g{};
+    g.status = status;
+    g.M = T; g.N = 3 * H; g.K = H;
+    g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_qkv);
+    g.out16 = qkv;
+    DIT_CUDA_TRY(ctx, launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st));
+    // attention
+    AttnParams ap{};
+    ap.out = a; ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
+    ap.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c.head_dim));
+    if (c.head_dim == 128) DIT_CUDA_TRY(ctx, launch_attention<128>(tm_qkv, ap, seq, st));
+    else DIT_CUDA_TRY(ctx, launch_attention<64>(tm_qkv, ap, seq, st));
+    // output projection + gate + residual
+    g = GemmParams{};
+    g.status = status;
+    g.M = T; g.N = H; g.K = H;
+    g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_o);
+    g.resid = stream; g.out32 = stream;
+    g.gate = modb + 2 * H; g.gate_stride = req_stride;
+    DIT_CUDA_TRY(ctx, launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st));
+    // LN2 + modulate
+    ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq);
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    // MLP up-projection + GELU-tanh
+    g = GemmParams{};
+    g.status = status;
+    g.M = T; g.N = F; g.K = H;
+    g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
+    g.out16 = u;
+    DIT_CUDA_TRY(ctx, launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st));
+    // MLP down-projection + gate + residual (last block writes the caller's output)
+    g = GemmParams{};
+    g.status = status;
+    g.M = T; g.N = H; g.K = F;
+    g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
+    g.resid = stream; g.out32 = (b == n_blocks - 1) ? out : stream;
+    g.gate = modb + 5 * H; g.gate_stride = req_stride;
+    DIT_CUDA_TRY(ctx, launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st));
+    launches += 7;
+  }
+  ctx->last_launches = launches;
+  ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
+  return DIT_OK;
+}
+
+dit_status check_step_args(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
+                           const float* out) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (n < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "n_requests is negative");
+  if (n == 0) return DIT_OK;
+  if (!tokens || !lens || !cond || !out) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  if (n > ctx->cfg.max_requests) return fail(ctx, DIT_ERR_CAPACITY, "n_requests exceeds max_requests");
+  if (n_blocks < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "n_blocks must be at least 1");
+  if (n_blocks > ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "n_blocks exceeds max_blocks");
+  long long total = 0;
+  for (int r = 0; r < n; ++r) {
+    if (lens[r] < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
+    total += lens[r];
+  }
+  if (total > ctx->cfg.max_total_tokens) return fail(ctx, DIT_ERR_CAPACITY, "packed batch exceeds max_total_tokens");
+  return DIT_OK;
+}
+
+}  // namespace
+
+// =============================================================================================== C ABI
+extern "C" {
+
+size_t dit_workspace_bytes(const dit_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(*cfg).bytes;
+}
+
+dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspace_bytes, dit_ctx** out) {
+  if (!out) return DIT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || !workspace) return DIT_ERR_INVALID_ARG;
+  if (!config_ok(cfg)) return DIT_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return DIT_ERR_INVALID_ARG;
+  const Layout lay = make_layout(*cfg);
+  if (workspace_bytes < lay.bytes) return DIT_ERR_CAPACITY;
+
+  int dev = 0, major = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DIT_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DIT_ERR_CUDA;
+  if (major != 10) return DIT_ERR_UNSUPPORTED_ARCH;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DIT_ERR_CUDA;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return DIT_ERR_CUDA;
+
+  dit_ctx* ctx = new (std::nothrow) dit_ctx();
+  if (!ctx) return DIT_ERR_INTERNAL;
+  ctx->cfg = *cfg;
+  ctx->lay = lay;
+  ctx->ws = static_cast<uint8_t*>(workspace);
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  ctx->num_sms = sms;
+  ctx->blocks = new (std::nothrow) BlockState[cfg->max_blocks];
+  ctx->last_launches = 0;
+  ctx->last_T = ctx->last_R = ctx->last_nb = 0;
+  ctx->err[0] = 0;
+  if (!ctx->blocks) { delete ctx; return DIT_ERR_INTERNAL; }
+
+  cudaError_t e = cudaSuccess;
+  auto opt_in = [&](const void* f, size_t bytes) {
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+  };
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&modulation_kernel), mod_smem_bytes(cfg->cond_dim));
+  if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
+  if (e != cudaSuccess) { delete[] ctx->blocks; delete ctx; return DIT_ERR_CUDA; }
+  *out = ctx;
+  return DIT_OK;
+}
+
+dit_status dit_ctx_destroy(dit_ctx* ctx) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  delete[] ctx->blocks;
+  delete ctx;
+  return DIT_OK;
+}
+
+dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weights* w, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (!w) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weights");
+  if (b < 0 || b >= ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "block index outside [0, max_blocks)");
+  if (!w->w_ada || !w->w_qkv || !w->w_o || !w->w_fc1 || !w->w_fc2) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weight matrix");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int H = ctx->cfg.hidden, F = ctx->cfg.mlp_hidden, C = ctx->cfg.cond_dim;
+  uint8_t* base = ctx->block_base(b);
+  const BlockLayout& L = ctx->lay.blk;
+  BlockState& bs = ctx->blocks[b];
+  bs.loaded = false;
+
+  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(base + L.w_ada, w->w_ada, static_cast<size_t>(C) * 6 * H * 2, cudaMemcpyDeviceToDevice, st));
+  auto bias = [&](const void* src, size_t off, int n) {
+    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + off), n);
+    return cudaGetLastError();
+  };
+  auto weight = [&](const void* src, size_t off, int K, int N) {   // [K, N] bf16 -> [N, K] fp16
+    dim3 grid((N + 31) / 32, (K + 31) / 32);
+    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    return cudaGetLastError();
+  };
+  DIT_CUDA_TRY(ctx, bias(w->b_ada, L.b_ada, 6 * H));
+  DIT_CUDA_TRY(ctx, weight(w->w_qkv, L.w_qkv, H, 3 * H));
+  DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
+  DIT_CUDA_TRY(ctx, weight(w->w_o, L.w_o, H, H));
+  DIT_CUDA_TRY(ctx, bias(w->b_o, L.b_o, H));
+  DIT_CUDA_TRY(ctx, weight(w->w_fc1, L.w_fc1, H, F));
+  DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
+  DIT_CUDA_TRY(ctx, weight(w->w_fc2, L.w_fc2, F, H));
+  DIT_CUDA_TRY(ctx, bias(w->b_fc2, L.b_fc2, H));
+
+  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN) ||
+      !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN) ||
+      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN) ||
+      !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+  bs.loaded = true;
+  return DIT_OK;
+}
+
+dit_status dit_pack_requests(const dit_request* reqs, int32_t n, int32_t* token_lens, int32_t* cu_seqlens,
+                             int32_t* row_req, int32_t* row_local, int32_t* total_tokens) {
+  if (n < 0 || (n > 0 && !reqs) || !token_lens || !cu_seqlens || !total_tokens) return DIT_ERR_INVALID_ARG;
+  long long cu = 0;
+  for (int r = 0; r < n; ++r) {
+    const dit_request& q = reqs[r];
+    if (q.height <= 0 || q.width <= 0 || q.height % 16 || q.width % 16 || q.n_text_tokens < 0) return DIT_ERR_SHAPE;
+    const long long l = static_cast<long long>(q.height / 16) * (q.width / 16) + q.n_text_tokens;
+    if (cu + l > INT32_MAX) return DIT_ERR_CAPACITY;
+    cu += l;
+  }
+  cu = 0;
+  cu_seqlens[0] = 0;
+  for (int r = 0; r < n; ++r) {
+    const int32_t l = (reqs[r].height / 16) * (reqs[r].width / 16) + reqs[r].n_text_tokens;
+    token_lens[r] = l;
+    for (int32_t i = 0; i < l; ++i) {
+      if (row_req) row_req[cu + i] = r;
+      if (row_local) row_local[cu + i] = i;
+    }
+    cu += l;
+    cu_seqlens[r + 1] = static_cast<int32_t>(cu);
+  }
+  *total_tokens = static_cast<int32_t>(cu);
+  return DIT_OK;
+}
+
+dit_status dit_pack_tokens(dit_ctx* ctx, const void* const* per_request_tokens, const int32_t* token_lens, int32_t n,
+                           void* packed_tokens, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (n < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "n is negative");
+  if (n == 0) return DIT_OK;
+  if (!per_request_tokens || !token_lens || !packed_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  if (n > ctx->cfg.max_requests) return fail(ctx, DIT_ERR_CAPACITY, "n exceeds max_requests");
+  SeqInfo seq{};
+  if (!build_seq(token_lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
+  PtrList pl{};
+  for (int r = 0; r < n; ++r) {
+    if (!per_request_tokens[r]) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL request buffer");
+    pl.ptr[r] = per_request_tokens[r];
+  }
+  const int row_vecs = ctx->cfg.hidden * 2 / 16;
+  const long long total = static_cast<long long>(seq.total) * row_vecs;
+  const int grid = static_cast<int>(std::min<long long>((total + 255) / 256, static_cast<long long>(ctx->num_sms) * 16));
+  pack_tokens_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(pl, seq, packed_tokens, row_vecs);
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
+  return DIT_OK;
+}
+
+dit_status dit_step_forward(dit_ctx* ctx, const void* packed_tokens, const int32_t* lens, int32_t n, const void* cond,
+                            int32_t n_blocks, float* out, void* stream) {
+  dit_status s = check_step_args(ctx, packed_tokens, lens, n, cond, n_blocks, out);
+  if (s != DIT_OK || n == 0) return s;
+  return step_impl(ctx, packed_tokens, lens, n, cond, n_blocks, out, static_cast<cudaStream_t>(stream));
+}
+
+dit_status dit_step_forward_host(dit_ctx* ctx, const void* host_tokens, const int32_t* lens, int32_t n,
+                                 const void* host_cond, int32_t n_blocks, float* host_out, void* stream) {
+  dit_status s = check_step_args(ctx, host_tokens, lens, n, host_cond, n_blocks, host_out);
+  if (s != DIT_OK || n == 0) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  size_t T = 0;
+  for (int r = 0; r < n; ++r) T += lens[r];
+  const size_t H = ctx->cfg.hidden, C = ctx->cfg.cond_dim;
+  void* d_tok = ctx->ws + ctx->lay.stage_tokens;
+  void* d_cond = ctx->ws + ctx->lay.stage_cond;
+  float* d_out = ctx->at<float>(ctx->lay.stage_out);
+  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(d_tok, host_tokens, T * H * 2, cudaMemcpyHostToDevice, st));
+  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(d_cond, host_cond, n * C * 2, cudaMemcpyHostToDevice, st));
+  s = step_impl(ctx, d_tok, lens, n, d_cond, n_blocks, d_out, st);
+  if (s != DIT_OK) return s;
+  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, d_out, T * H * 4, cudaMemcpyDeviceToHost, st));
+  DIT_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  return DIT_OK;
+}
+
+dit_status dit_ctx_poll_status(dit_ctx* ctx) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  int word[4] = {0, 0, 0, 0};
+  DIT_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  DIT_CUDA_TRY(ctx, cudaMemcpy(word, ctx->ws + ctx->lay.status, sizeof(word), cudaMemcpyDeviceToHost));
+  if (word[0] == kStatusOk) return DIT_OK;
+  DIT_CUDA_TRY(ctx, cudaMemset(ctx->ws + ctx->lay.status, 0, sizeof(word)));
+  return fail(ctx, DIT_ERR_TIMEOUT, "a bounded wait ran out in the %s kernel", word[0] == kStatusGemmTimeout ? "GEMM" : "attention");
+}
+
+dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t* rows, int64_t* cols, int32_t* elem_bytes) {
+  if (!ctx || !ptr || !rows || !cols || !elem_bytes) return DIT_ERR_INVALID_ARG;
+  const int64_t H = ctx->cfg.hidden, F = ctx->cfg.mlp_hidden, T = ctx->last_T;
+  switch (which) {
+    case DIT_TAP_H: *ptr = ctx->ws + ctx->lay.h; *rows = T; *cols = H; *elem_bytes = 2; break;
+    case DIT_TAP_QKV: *ptr = ctx->ws + ctx->lay.qkv; *rows = T; *cols = 3 * H; *elem_bytes = 2; break;
+    case DIT_TAP_ATTN: *ptr = ctx->ws + ctx->lay.a; *rows = T; *cols = H; *elem_bytes = 2; break;
+    case DIT_TAP_U: *ptr = ctx->ws + ctx->lay.u; *rows = T; *cols = F; *elem_bytes = 2; break;
+    case DIT_TAP_MOD: *ptr = ctx->ws + ctx->lay.mod; *rows = static_cast<int64_t>(ctx->last_R) * ctx->last_nb; *cols = 6 * H; *elem_bytes = 4; break;
+    case DIT_TAP_STREAM: *ptr = ctx->ws + ctx->lay.stream; *rows = T; *cols = H; *elem_bytes = 4; break;
+    default: return DIT_ERR_INVALID_ARG;
+  }
+  return DIT_OK;
+}
+
+int64_t dit_last_launch_count(const dit_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+const char* dit_status_string(dit_status s) {
+  switch (s) {
+    case DIT_OK: return "ok";
+    case DIT_ERR_INVALID_ARG: return "invalid argument";
+    case DIT_ERR_SHAPE: return "unsupported shape";
+    case DIT_ERR_CAPACITY: return "capacity exceeded";
+    case DIT_ERR_NOT_LOADED: return "block weights not loaded";
+    case DIT_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    case DIT_ERR_CUDA: return "CUDA error";
+    case DIT_ERR_TIMEOUT: return "device wait timed out";
+    case DIT_ERR_INTERNAL: return "internal error";
+  }
+  return "unknown status";
+}
+
+const char* dit_last_error(const dit_ctx* ctx) { return ctx ? ctx->err : ""; }
+
+}  // extern "C"

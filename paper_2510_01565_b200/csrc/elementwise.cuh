@@ -1,0 +1,206 @@
+// HBM-bound kernels of the step: adaLN modulation GEMV, LayerNorm + modulate, token gather,
+// and the one-off weight re-layout done at load time.
+#pragma once
+#include "common.cuh"
+
+namespace dit {
+
+// ------------------------------------------------------------------------------------------------
+// adaLN modulation for all blocks at once:
+//   mod[r, b, j] = sum_c SiLU(cond[r, c]) * W_ada_b[c, j] + b_ada_b[j],   j in [0, 6H)
+// Bound by reading W_ada once (C x 6H bf16 per block).  A CTA owns 256 consecutive columns of one
+// block: 32 column groups (8 bf16 = 16 B per load) x 8 slices of the C range; slice partials are
+// combined in shared memory in slice order, so the result does not depend on the number of requests.
+// Requests are processed in groups of kModReqGroup to bound registers.
+// ------------------------------------------------------------------------------------------------
+constexpr int kModReqGroup = 8;
+constexpr int kModThreads = 256;
+constexpr int kModCols = 256;
+
+struct ModParams {
+  const __nv_bfloat16* cond;     // [R, C]
+  const __nv_bfloat16* w_ada0;   // block 0's W_ada [C, 6H]; block b at + b * w_block_stride (elements)
+  const float* b_ada0;           // block 0's bias [6H] fp32; block b at + b * b_block_stride
+  long long w_block_stride, b_block_stride;
+  float* mod;                    // [R, NB, 6H]
+  int R, C, N6, NB;
+};
+
+__global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams p) {
+  extern __shared__ float sm[];                       // silu(cond) [G][C], then partials [8][G][256]
+  const int cols_per_block = (p.N6 + kModCols - 1) / kModCols;
+  const int blk = blockIdx.x / cols_per_block;
+  const int col_base = (blockIdx.x % cols_per_block) * kModCols;
+  const int cg = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  const int col = col_base + cg * 8;
+  const __nv_bfloat16* w = p.w_ada0 + blk * p.w_block_stride;
+  const float* bias = p.b_ada0 + blk * p.b_block_stride;
+  float* s_act = sm;
+  float* s_part = sm + kModReqGroup * p.C;
+  const int c_per = (p.C + 7) / 8;
+  const int c0 = slice * c_per, c1 = min(p.C, c0 + c_per);
+
+  for (int r0 = 0; r0 < p.R; r0 += kModReqGroup) {
+    const int g = min(kModReqGroup, p.R - r0);
+    __syncthreads();
+    for (int i = threadIdx.x; i < kModReqGroup * p.C; i += kModThreads) {
+      const int rr = i / p.C, cc = i % p.C;
+      float v = 0.f;
+      if (rr < g) {
+        const float x = __bfloat162float(p.cond[static_cast<size_t>(r0 + rr) * p.C + cc]);
+        v = x / (1.0f + __expf(-x));
+      }
+      s_act[i] = v;
+    }
+    __syncthreads();
+    float acc[kModReqGroup][8];
+#pragma unroll
+    for (int rr = 0; rr < kModReqGroup; ++rr)
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[rr][k] = 0.f;
+    if (col < p.N6) {
+#pragma unroll 4
+      for (int c = c0; c < c1; ++c) {
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(w + static_cast<size_t>(c) * p.N6 + col));
+        const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+        float wf[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          wf[2 * k] = __uint_as_float(u[k] << 16);
+          wf[2 * k + 1] = __uint_as_float(u[k] & 0xFFFF0000u);
+        }
+#pragma unroll
+        for (int rr = 0; rr < kModReqGroup; ++rr) {
+          const float a = s_act[rr * p.C + c];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) acc[rr][k] = fmaf(a, wf[k], acc[rr][k]);
+        }
+      }
+    }
+#pragma unroll
+    for (int rr = 0; rr < kModReqGroup; ++rr)
+#pragma unroll
+      for (int k = 0; k < 8; ++k) s_part[(slice * kModReqGroup + rr) * kModCols + cg * 8 + k] = acc[rr][k];
+    __syncthreads();
+    for (int i = threadIdx.x; i < g * kModCols; i += kModThreads) {
+      const int rr = i / kModCols, cc = i % kModCols;
+      if (col_base + cc < p.N6) {
+        float v = 0.f;
+#pragma unroll
+        for (int sl = 0; sl < 8; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModCols + cc];
+        p.mod[(static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc] = v + bias[col_base + cc];
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// LayerNorm (over H, biased variance, eps inside the root, no affine) + adaLN modulate:
+//   h[row, :] = (x - mean) * rstd * (1 + scale[req]) + shift[req]        -> fp16
+// One warp per row, the row held in registers (H <= 4096), two-pass statistics, fixed shuffle order.
+// kFromBf16 = true reads the packed bf16 tokens (first block) and also writes the fp32 residual stream.
+// ------------------------------------------------------------------------------------------------
+constexpr int kLnWarps = 8;
+constexpr int kLnMaxVec = 32;   // float4 per lane: H <= 32 * 32 * 4 = 4096
+
+template <bool kFromBf16>
+__global__ void __launch_bounds__(kLnWarps * 32)
+ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
+                   const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
+                   int T, int H, float eps, const __grid_constant__ SeqInfo seq) {
+  const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= T) return;
+  const int nvec = H >> 2;
+  float4 v[kLnMaxVec];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxVec; ++i) {
+    const int idx = i * 32 + lane;
+    if (idx < nvec) {
+      if (kFromBf16) {
+        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(xin) + static_cast<size_t>(row) * H) + idx);
+        v[i] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+        reinterpret_cast<float4*>(stream_out + static_cast<size_t>(row) * H)[idx] = v[i];
+      } else {
+        v[i] = reinterpret_cast<const float4*>(static_cast<const float*>(xin) + static_cast<size_t>(row) * H)[idx];
+      }
+      sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum / static_cast<float>(H);
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxVec; ++i) {
+    if (i * 32 + lane < nvec) {
+      const float a = v[i].x - mean, b = v[i].y - mean, c = v[i].z - mean, d = v[i].w - mean;
+      sq += (a * a + b * b) + (c * c + d * d);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  const float rstd = rsqrtf(sq / static_cast<float>(H) + eps);
+  const int req = find_request(seq, row);
+  const float4* sh = reinterpret_cast<const float4*>(shift0 + req * req_stride);
+  const float4* sc = reinterpret_cast<const float4*>(scale0 + req * req_stride);
+  uint2* dst = reinterpret_cast<uint2*>(h + static_cast<size_t>(row) * H);
+#pragma unroll
+  for (int i = 0; i < kLnMaxVec; ++i) {
+    const int idx = i * 32 + lane;
+    if (idx < nvec) {
+      const float4 s1 = __ldg(sc + idx), s0 = __ldg(sh + idx);
+      const float a = (v[i].x - mean) * rstd * (1.f + s1.x) + s0.x;
+      const float b = (v[i].y - mean) * rstd * (1.f + s1.y) + s0.y;
+      const float c = (v[i].z - mean) * rstd * (1.f + s1.z) + s0.z;
+      const float d = (v[i].w - mean) * rstd * (1.f + s1.w) + s0.w;
+      const __half2 lo = __floats2half2_rn(a, b), hi = __floats2half2_rn(c, d);
+      dst[idx] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Token gather: per-request [L_r, H] bf16 buffers -> one packed [T, H] bf16 buffer (16-byte copies).
+// ------------------------------------------------------------------------------------------------
+struct PtrList { const void* ptr[DIT_MAX_REQUESTS]; };
+
+__global__ void __launch_bounds__(256)
+pack_tokens_kernel(const __grid_constant__ PtrList src, const __grid_constant__ SeqInfo seq, void* __restrict__ dst, int row_vecs) {
+  const long long total = static_cast<long long>(seq.total) * row_vecs;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+    const int row = static_cast<int>(i / row_vecs), vcol = static_cast<int>(i % row_vecs);
+    const int r = find_request(seq, row);
+    const uint4* s = static_cast<const uint4*>(src.ptr[r]) + static_cast<size_t>(row - seq.cu[r]) * row_vecs + vcol;
+    static_cast<uint4*>(dst)[i] = __ldg(s);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Weight load: bf16 [K, N] row-major -> fp16 [N, K] row-major (K-major B operand of the GEMMs).
+// bf16 -> fp16 is exact for |w| >= 2^-17 (8 significant bits fit fp16's normal and subnormal range).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+transpose_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __restrict__ out, int K, int N) {
+  __shared__ float tile[32][33];
+  const int n0 = blockIdx.x * 32, k0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+  for (int i = ty; i < 32; i += 8) {
+    const int k = k0 + i, n = n0 + tx;
+    tile[i][tx] = (k < K && n < N) ? __bfloat162float(in[static_cast<size_t>(k) * N + n]) : 0.f;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int n = n0 + i, k = k0 + tx;
+    if (n < N && k < K) out[static_cast<size_t>(n) * K + k] = __float2half_rn(tile[tx][i]);
+  }
+}
+
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = in ? __bfloat162float(in[i]) : 0.f;
+}
+
+}  // namespace dit

@@ -1,0 +1,216 @@
+// Persistent warp-specialised GEMM for sm_100a:  C[M,N] = A[M,K] * Wt[N,K]^T  (+ fused epilogue).
+//
+// A (activations, fp16, row-major [M,K]) and Wt (weights, fp16, row-major [N,K]) are both K-major.
+// TMA brings 128x64 (A) and 256x64 (Wt) tiles with the 128-byte swizzle into a 4-stage shared-memory
+// ring; one thread issues tcgen05.mma (128x256x16, kind::f16, fp32 accumulate) into one of two TMEM
+// accumulators (2 x 256 columns), so that the epilogue of a tile overlaps the main loop of the next.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue (one TMEM lane
+// quarter each).  Tiles are taken in a fixed order and every output element is accumulated over K in
+// the same order whatever M is: a row's result does not depend on where it sits in the batch.
+//
+// Epilogues (the fused parts of the adaLN-Zero block):
+//   kEpiBiasF16      out16 = acc + bias                                   (QKV projection)
+//   kEpiBiasGeluF16  out16 = gelu_tanh(acc + bias)                        (MLP up-projection)
+//   kEpiGateResidF32 out32 = resid + gate[request(row)] * (acc + bias)    (attention / MLP output)
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace dit {
+
+enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32 = 2 };
+
+struct GemmParams {
+  int M, N, K;
+  const float* bias;        // [N]
+  __half* out16;            // [M, N]
+  const float* resid;       // [M, N]
+  float* out32;             // [M, N]
+  const float* gate;        // gate vector of request 0 for this block; request r at gate + r * gate_stride
+  long long gate_stride;
+  int* status;              // device status word
+};
+
+namespace gemm_cfg {
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+}  // namespace gemm_cfg
+
+__device__ __forceinline__ float gelu_tanh_f32(float z) {
+  const float k0 = 0.7978845608028654f, k1 = 0.044715f;
+  float y = k0 * (z + k1 * z * z * z);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(y));
+  return 0.5f * z * (1.0f + t);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(gemm_cfg::THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const GemmParams p, const __grid_constant__ SeqInfo seq) {
+  using namespace gemm_cfg;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
+  // bars: [0,S) full, [S,2S) empty, [2S,2S+2) tmem_full, [2S+2,2S+4) tmem_empty
+  const uint32_t bar0 = base + STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_m = (p.M + BM - 1) / BM, num_n = (p.N + BN - 1) / BN;
+  const int num_tiles = num_m * num_n;
+  const int num_k = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) { prefetch_tmap(&tmA); prefetch_tmap(&tmB); }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) goto done;
+          mbar_arrive_expect_tx(full_bar(stage), STAGE_BYTES);
+          const uint32_t sa = base + stage * STAGE_BYTES;
+          tma_load_2d(sa, &tmA, kb * BK, m0, full_bar(stage));
+          tma_load_2d(sa + A_BYTES, &tmB, kb * BK, n0, full_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_f16(BM, BN, false);
+      int stage = 0; uint32_t phase = 0; int it = 0;
+      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+        const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) goto done;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) goto done;
+          tc_fence_after();
+          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa, 16, 1024);
+          const uint64_t bdesc = smem_desc_sw128(sa + A_BYTES, 16, 1024);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)   // 32 bytes further along K inside the swizzled row
+            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          umma_commit(empty_bar(stage));       // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        umma_commit(tfull_bar(acc));           // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps)
+    const int quarter = warp & 3;              // TMEM lanes this warp may read: [32*quarter, +32)
+    int it = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+      const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
+      const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      const float* gate_row = nullptr;
+      if (EPI == kEpiGateResidF32 && row_ok) gate_row = p.gate + find_request(seq, row) * p.gate_stride;
+      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        __syncwarp();                          // tcgen05.ld is warp-collective: reconverge first
+        tmem_ld32(t_row + c * 32, r);
+        tmem_ld_wait();
+        const int col0 = n0 + c * 32;
+        const bool full = (col0 + 32 <= p.N);
+        if (!row_ok || col0 >= p.N) {
+          // nothing to store for this lane / chunk
+        } else if (EPI == kEpiGateResidF32) {
+          const float* res = p.resid + static_cast<size_t>(row) * p.N + col0;
+          float* dst = p.out32 + static_cast<size_t>(row) * p.N + col0;
+          if (full) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col0) + v);
+              const float4 g = __ldg(reinterpret_cast<const float4*>(gate_row + col0) + v);
+              const float4 x = *(reinterpret_cast<const float4*>(res) + v);
+              float4 o;
+              o.x = x.x + g.x * (__uint_as_float(r[4 * v + 0]) + b.x);
+              o.y = x.y + g.y * (__uint_as_float(r[4 * v + 1]) + b.y);
+              o.z = x.z + g.z * (__uint_as_float(r[4 * v + 2]) + b.z);
+              o.w = x.w + g.w * (__uint_as_float(r[4 * v + 3]) + b.w);
+              *(reinterpret_cast<float4*>(dst) + v) = o;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i < p.N) dst[i] = res[i] + gate_row[col0 + i] * (__uint_as_float(r[i]) + p.bias[col0 + i]);
+          }
+        } else {
+          __half* dst = p.out16 + static_cast<size_t>(row) * p.N + col0;
+          if (full) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const int i = 8 * v + 2 * h;
+                float a = __uint_as_float(r[i]) + __ldg(p.bias + col0 + i);
+                float b = __uint_as_float(r[i + 1]) + __ldg(p.bias + col0 + i + 1);
+                if (EPI == kEpiBiasGeluF16) { a = gelu_tanh_f32(a); b = gelu_tanh_f32(b); }
+                const __half2 hh = __floats2half2_rn(a, b);
+                w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+              *(reinterpret_cast<uint4*>(dst) + v) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              if (col0 + i < p.N) {
+                float a = __uint_as_float(r[i]) + p.bias[col0 + i];
+                if (EPI == kEpiBiasGeluF16) a = gelu_tanh_f32(a);
+                dst[i] = __float2half_rn(a);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+
+done:
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+  if (threadIdx.x == 0 && *abort_flag) atomicMax(p.status, kStatusGemmTimeout);
+}
+
+}  // namespace dit
