@@ -59,11 +59,11 @@ typedef enum {
 } dit_status;
 
 typedef struct {
-  int32_t hidden;           /* H; multiple of 64, <= 8192 */
+  int32_t hidden;           /* H; multiple of 64, <= 4096 */
   int32_t n_heads;          /* nh; H = nh * head_dim */
   int32_t head_dim;         /* d; 64 or 128 */
   int32_t mlp_hidden;       /* F; multiple of 64 */
-  int32_t cond_dim;         /* C; multiple of 8 */
+  int32_t cond_dim;         /* C; 1..4096 */
   int32_t max_blocks;       /* weight slots carved from the workspace */
   int32_t max_total_tokens; /* capacity T_max of one packed batch */
   int32_t max_requests;     /* capacity R_max, <= DIT_MAX_REQUESTS */
@@ -149,6 +149,18 @@ dit_status dit_ctx_poll_status(dit_ctx *ctx);
 typedef enum { DIT_TAP_H = 0, DIT_TAP_QKV = 1, DIT_TAP_ATTN = 2, DIT_TAP_U = 3, DIT_TAP_MOD = 4, DIT_TAP_STREAM = 5 } dit_tap;
 dit_status dit_debug_tap(dit_ctx *ctx, dit_tap which, const void **ptr, int64_t *rows, int64_t *cols,
                          int32_t *elem_bytes);
+
+/* Per-kernel timing for benchmarks.  While enabled, every kernel launch of a step is bracketed by
+ * a pair of CUDA events on the step's stream (events are created on demand and kept; no device
+ * memory is allocated).  dit_ctx_read_timing synchronises the device, adds up the elapsed time and
+ * the number of launches per kernel kind since the last read (HOST arrays of DIT_KERNEL_KINDS
+ * entries) and starts a new accumulation. */
+typedef enum {
+  DIT_KERNEL_MODULATION = 0, DIT_KERNEL_LN_MODULATE = 1, DIT_KERNEL_GEMM_QKV = 2, DIT_KERNEL_ATTENTION = 3,
+  DIT_KERNEL_GEMM_PROJ = 4, DIT_KERNEL_GEMM_FC1 = 5, DIT_KERNEL_GEMM_FC2 = 6, DIT_KERNEL_KINDS = 7
+} dit_kernel_kind;
+dit_status dit_ctx_set_timing(dit_ctx *ctx, int32_t enabled);
+dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *launches_by_kernel);
 
 /* Number of kernel launches issued by the last dit_step_forward on this context. */
 int64_t dit_last_launch_count(const dit_ctx *ctx);

@@ -18,11 +18,12 @@ LIB_PATH = os.path.join(HERE, "libdit.so")
 DIT_OK = 0
 STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
                 "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
+KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_host",
-           "dit_ctx_poll_status", "dit_debug_tap", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
 
 class DitConfig(C.Structure):
@@ -82,6 +83,10 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_poll_status.argtypes = [vp]
     lib.dit_debug_tap.restype = C.c_int
     lib.dit_debug_tap.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+    lib.dit_ctx_set_timing.restype = C.c_int
+    lib.dit_ctx_set_timing.argtypes = [vp, i32]
+    lib.dit_ctx_read_timing.restype = C.c_int
+    lib.dit_ctx_read_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.dit_last_launch_count.restype = i64
     lib.dit_last_launch_count.argtypes = [vp]
     lib.dit_status_string.restype = C.c_char_p
@@ -224,6 +229,15 @@ class DitContext:
 
     def dit_ctx_poll_status(self):
         self._check(self.lib.dit_ctx_poll_status(self.handle))
+
+    def dit_ctx_set_timing(self, enabled: bool):
+        self._check(self.lib.dit_ctx_set_timing(self.handle, 1 if enabled else 0))
+
+    def dit_ctx_read_timing(self) -> Dict[str, Dict[str, float]]:
+        ms = (C.c_double * len(KERNEL_KINDS))()
+        n = (C.c_int64 * len(KERNEL_KINDS))()
+        self._check(self.lib.dit_ctx_read_timing(self.handle, ms, n))
+        return {k: {"ms": ms[i], "launches": int(n[i])} for i, k in enumerate(KERNEL_KINDS)}
 
     def dit_last_launch_count(self) -> int:
         return int(self.lib.dit_last_launch_count(self.handle))

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "attention.cuh"
 #include "common.cuh"
@@ -92,6 +93,11 @@ struct dit_ctx {
   int64_t last_launches;
   int last_T, last_R, last_nb;
   char err[256];
+  // optional per-kernel timing (CUDA events recorded around every launch of a step)
+  bool timing;
+  std::vector<cudaEvent_t> ev_pool;        // pairs: [2i] start, [2i+1] stop
+  std::vector<int> ev_kind;                // kind of pair i
+  size_t ev_used;                          // pairs recorded since the last read
 
   template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   uint8_t* block_base(int b) const { return ws + lay.weights + lay.blk.bytes * static_cast<size_t>(b); }
@@ -180,6 +186,27 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
 
   int64_t launches = 0;
   const long long req_stride = static_cast<long long>(n_blocks) * 6 * H;
+  // Runs one launch; with timing enabled, brackets it with a pair of events on the stream.
+  auto timed = [&](int kind, auto&& launch) -> cudaError_t {
+    ++launches;
+    if (!ctx->timing) return launch();
+    if (ctx->ev_used * 2 + 2 > ctx->ev_pool.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e;
+        cudaError_t ce = cudaEventCreate(&e);
+        if (ce != cudaSuccess) return ce;
+        ctx->ev_pool.push_back(e);
+      }
+      ctx->ev_kind.push_back(kind);
+    }
+    const size_t i = ctx->ev_used++;
+    ctx->ev_kind[i] = kind;
+    cudaError_t ce = cudaEventRecord(ctx->ev_pool[2 * i], st);
+    if (ce != cudaSuccess) return ce;
+    ce = launch();
+    if (ce != cudaSuccess) return ce;
+    return cudaEventRecord(ctx->ev_pool[2 * i + 1], st);
+  };
 
   {  // adaLN modulation vectors of every block
     ModParams mp{};
@@ -190,9 +217,10 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     mp.b_block_stride = static_cast<long long>(ctx->lay.blk.bytes / 4);
     mp.mod = mod; mp.R = n; mp.C = c.cond_dim; mp.N6 = 6 * H; mp.NB = n_blocks;
     const int grid = n_blocks * ((6 * H + kModCols - 1) / kModCols);
-    modulation_kernel<<<grid, kModThreads, mod_smem_bytes(c.cond_dim), st>>>(mp);
-    DIT_CUDA_TRY(ctx, cudaGetLastError());
-    ++launches;
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_MODULATION, [&] {
+      modulation_kernel<<<grid, kModThreads, mod_smem_bytes(c.cond_dim), st>>>(mp);
+      return cudaGetLastError();
+    }));
   }
 
   const int ln_grid = (T + kLnWarps - 1) / kLnWarps;
@@ -201,24 +229,27 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     const uint8_t* wb = ctx->block_base(b);
     const float* modb = mod + static_cast<size_t>(b) * 6 * H;   // request 0; request r at + r * req_stride
     // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
-    if (b == 0)
-      ln_modulate_kernel<true><<<ln_grid, kLnWarps * 32, 0, st>>>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
-    else
-      ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
-    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
+      if (b == 0)
+        ln_modulate_kernel<true><<<ln_grid, kLnWarps * 32, 0, st>>>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
+      else
+        ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
+      return cudaGetLastError();
+    }));
     // QKV projection
     GemmParams g{};
     g.status = status;
     g.M = T; g.N = 3 * H; g.K = H;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_qkv);
     g.out16 = qkv;
-    DIT_CUDA_TRY(ctx, launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st));
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] { return launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st); }));
     // attention
     AttnParams ap{};
     ap.out = a; ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
     ap.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c.head_dim));
-    if (c.head_dim == 128) DIT_CUDA_TRY(ctx, launch_attention<128>(tm_qkv, ap, seq, st));
-    else DIT_CUDA_TRY(ctx, launch_attention<64>(tm_qkv, ap, seq, st));
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_ATTENTION, [&] {
+      return c.head_dim == 128 ? launch_attention<128>(tm_qkv, ap, seq, st) : launch_attention<64>(tm_qkv, ap, seq, st);
+    }));
     // output projection + gate + residual
     g = GemmParams{};
     g.status = status;
@@ -226,17 +257,19 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_o);
     g.resid = stream; g.out32 = stream;
     g.gate = modb + 2 * H; g.gate_stride = req_stride;
-    DIT_CUDA_TRY(ctx, launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st));
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st); }));
     // LN2 + modulate
-    ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq);
-    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
+      ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq);
+      return cudaGetLastError();
+    }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};
     g.status = status;
     g.M = T; g.N = F; g.K = H;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
     g.out16 = u;
-    DIT_CUDA_TRY(ctx, launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st));
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st); }));
     // MLP down-projection + gate + residual (last block writes the caller's output)
     g = GemmParams{};
     g.status = status;
@@ -244,8 +277,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
     g.resid = stream; g.out32 = (b == n_blocks - 1) ? out : stream;
     g.gate = modb + 5 * H; g.gate_stride = req_stride;
-    DIT_CUDA_TRY(ctx, launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st));
-    launches += 7;
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st); }));
   }
   ctx->last_launches = launches;
   ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
@@ -312,6 +344,8 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->blocks = new (std::nothrow) BlockState[cfg->max_blocks];
   ctx->last_launches = 0;
   ctx->last_T = ctx->last_R = ctx->last_nb = 0;
+  ctx->timing = false;
+  ctx->ev_used = 0;
   ctx->err[0] = 0;
   if (!ctx->blocks) { delete ctx; return DIT_ERR_INTERNAL; }
 
@@ -333,6 +367,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
 
 dit_status dit_ctx_destroy(dit_ctx* ctx) {
   if (!ctx) return DIT_ERR_INVALID_ARG;
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   delete[] ctx->blocks;
   delete ctx;
   return DIT_OK;
@@ -479,6 +514,27 @@ dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t*
     case DIT_TAP_STREAM: *ptr = ctx->ws + ctx->lay.stream; *rows = T; *cols = H; *elem_bytes = 4; break;
     default: return DIT_ERR_INVALID_ARG;
   }
+  return DIT_OK;
+}
+
+dit_status dit_ctx_set_timing(dit_ctx* ctx, int32_t enabled) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->timing = enabled != 0;
+  ctx->ev_used = 0;
+  return DIT_OK;
+}
+
+dit_status dit_ctx_read_timing(dit_ctx* ctx, double* ms_by_kernel, int64_t* launches_by_kernel) {
+  if (!ctx || !ms_by_kernel || !launches_by_kernel) return DIT_ERR_INVALID_ARG;
+  for (int k = 0; k < DIT_KERNEL_KINDS; ++k) { ms_by_kernel[k] = 0.0; launches_by_kernel[k] = 0; }
+  DIT_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  for (size_t i = 0; i < ctx->ev_used; ++i) {
+    float ms = 0.f;
+    DIT_CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->ev_pool[2 * i], ctx->ev_pool[2 * i + 1]));
+    ms_by_kernel[ctx->ev_kind[i]] += ms;
+    launches_by_kernel[ctx->ev_kind[i]] += 1;
+  }
+  ctx->ev_used = 0;
   return DIT_OK;
 }
 

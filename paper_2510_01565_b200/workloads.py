@@ -191,8 +191,13 @@ def _draw(name, dims, n_blocks, reqs, rng, timestep_cond, with_weights) -> Workl
 
 
 def make_workload(name: str, seed: int = 0, n_blocks: int | None = None,
-                  with_weights: bool = True) -> Workload:
-    """One of the five benchmark configurations, fully seeded."""
+                  with_weights: bool = True, n_blocks_drawn: int | None = None) -> Workload:
+    """One of the five benchmark configurations, fully seeded.
+
+    `n_blocks_drawn` draws only the first few blocks' weights (they come last in the draw order,
+    so the requests, tokens, cond vectors and those blocks are unchanged) while `n_blocks` keeps
+    the configuration's depth.
+    """
     dims, nb, reqs = CONFIGS[name]
     nb = nb if n_blocks is None else n_blocks
     rng = np.random.default_rng(seed)
@@ -201,4 +206,7 @@ def make_workload(name: str, seed: int = 0, n_blocks: int | None = None,
         reqs = [(r, 512) for r in res]
     reqs3 = [(r, r, n_text) for (r, n_text) in reqs]
     # config 1 draws its cond vector directly; the large configs add a timestep embedding
-    return _draw(name, dims, nb, reqs3, rng, timestep_cond=(dims is LARGE), with_weights=with_weights)
+    wl = _draw(name, dims, nb if n_blocks_drawn is None else min(nb, n_blocks_drawn), reqs3, rng,
+               timestep_cond=(dims is LARGE), with_weights=with_weights)
+    wl.n_blocks = nb
+    return wl
