@@ -153,11 +153,11 @@ def run_gpu(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2510_01565_b200 import replicas
     dist = None
     if world > 1:
-        import torch.distributed as dist
         torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = replicas.init_process_group("nccl", torch.device("cuda", local_rank))
     else:
         torch.cuda.set_device(0)
     build.build_library()
@@ -179,11 +179,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms: float) -> float:
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(ms, dist, "cuda")
 
     # ---------------------------------------------------------------- device-resident throughput
     for _ in range(args.warmup):
@@ -208,7 +204,7 @@ def run_gpu(args):
     launches = ctx.dit_last_launch_count() * args.steps
     ms_step = ms_total / args.steps
     img_tokens = wl.image_tokens * world
-    value = img_tokens / (ms_step * 1e-3)
+    value = replicas.whole_job_rate(wl.image_tokens, world, ms_step)
     flops = wl.flops_per_step()
     tflops = flops / (ms_step * 1e-3) / 1e12
 
