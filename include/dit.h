@@ -162,6 +162,25 @@ typedef enum {
 dit_status dit_ctx_set_timing(dit_ctx *ctx, int32_t enabled);
 dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *launches_by_kernel);
 
+/* adaLN modulation vectors with no allocation at all (the paper has no counterpart; this exists for
+ * hosts that cannot allocate device memory: a plugin called inside another runtime's execution
+ * phase, a process whose memory pool belongs to a framework, a caller that was handed fixed buffers
+ * and nothing else).  It needs no context and no workspace.
+ *   mod_out[r, :] = W_ada^T SiLU(cond[r, :]) + b_ada        device [n_requests, 6H] fp32
+ *   cond device [n_requests, C] bf16; w_ada device [C, 6H] bf16; b_ada device [6H] bf16 or NULL (zero)
+ * The result equals the `mod` vectors dit_step_forward computes for that block.  The fp32 copy of
+ * the bias, which the context path keeps in the caller's workspace, lives here in a fixed 96 KiB
+ * array inside the library image (every GPU that loads the library holds it until the process
+ * exits).  Limits: hidden a multiple of 64 and <= 4096, cond_dim <= 4096, n_requests <=
+ * DIT_MAX_REQUESTS; anything larger returns DIT_ERR_CAPACITY, an unsupported hidden DIT_ERR_SHAPE,
+ * and nothing is launched.  The first call on a device looks the array's device address up and
+ * raises the kernel's shared-memory limit; make that first call outside any stream capture.  All
+ * calls share the one array, which keeps the previous call's bias until the next call rewrites
+ * it (zeros for a NULL bias), so two calls whose kernels overlap on the GPU (different streams)
+ * race: issue calls on one stream, or order them with events.  Asynchronous on `stream`. */
+dit_status dit_modulation_noalloc(const void *cond, const void *w_ada, const void *b_ada, int32_t n_requests,
+                                  int32_t cond_dim, int32_t hidden, float *mod_out, void *stream);
+
 /* Number of kernel launches issued by the last dit_step_forward on this context. */
 int64_t dit_last_launch_count(const dit_ctx *ctx);
 

@@ -23,7 +23,7 @@ TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_host",
-           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
 
 class DitConfig(C.Structure):
@@ -87,6 +87,8 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_set_timing.argtypes = [vp, i32]
     lib.dit_ctx_read_timing.restype = C.c_int
     lib.dit_ctx_read_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.dit_modulation_noalloc.restype = C.c_int
+    lib.dit_modulation_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     lib.dit_last_launch_count.restype = i64
     lib.dit_last_launch_count.argtypes = [vp]
     lib.dit_status_string.restype = C.c_char_p
@@ -253,6 +255,28 @@ class DitContext:
         torch.cuda.synchronize()
         flat = self.workspace[(base - self.workspace.data_ptr()) + off:(base - self.workspace.data_ptr()) + off + rows.value * cols.value * eb.value]
         return flat.view(dtype).view(rows.value, cols.value).clone()
+
+
+def dit_modulation_noalloc(cond, w_ada, b_ada, mod_out, stream=None):
+    """cond [R,C], w_ada [C,6H], b_ada [6H] or None: CUDA bf16 tensors; mod_out [R,6H] CUDA fp32, written in place.
+
+    Marshalling only: the caller provides every buffer, nothing is allocated here or in the library.
+    """
+    import torch
+    lib = load_library()
+    R, Cd = cond.shape
+    H = w_ada.shape[1] // 6
+    assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous()
+    assert w_ada.is_cuda and w_ada.dtype == torch.bfloat16 and w_ada.is_contiguous() and w_ada.shape == (Cd, 6 * H)
+    assert b_ada is None or (b_ada.is_cuda and b_ada.dtype == torch.bfloat16 and b_ada.shape == (6 * H,))
+    assert mod_out.is_cuda and mod_out.dtype == torch.float32 and mod_out.is_contiguous() and mod_out.shape == (R, 6 * H)
+    s = torch.cuda.current_stream() if stream is None else stream
+    st = lib.dit_modulation_noalloc(C.c_void_p(cond.data_ptr()), C.c_void_p(w_ada.data_ptr()),
+                                    C.c_void_p(b_ada.data_ptr()) if b_ada is not None else None, R, Cd, H,
+                                    C.c_void_p(mod_out.data_ptr()), C.c_void_p(s.cuda_stream))
+    if st != DIT_OK:
+        raise DitError(st, lib.dit_status_string(st).decode())
+    return mod_out
 
 
 def context_for(dims, max_blocks: int, max_total_tokens: int, max_requests: int = 8) -> DitContext:

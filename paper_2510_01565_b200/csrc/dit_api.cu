@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -19,6 +20,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr size_t kAlign = 1024;
+constexpr int kMaxCondDim = 4096;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets (bytes) inside one block's weight slot.
@@ -37,7 +39,7 @@ bool config_ok(const dit_config* c) {
   if (c->head_dim != 64 && c->head_dim != 128) return false;
   if (c->n_heads < 1 || static_cast<long long>(c->n_heads) * c->head_dim != c->hidden) return false;
   if (c->mlp_hidden < 64 || c->mlp_hidden % 64) return false;
-  if (c->cond_dim < 1 || c->cond_dim > 4096) return false;
+  if (c->cond_dim < 1 || c->cond_dim > kMaxCondDim) return false;
   if (c->max_blocks < 1 || c->max_total_tokens < 1) return false;
   if (c->max_requests < 1 || c->max_requests > DIT_MAX_REQUESTS) return false;
   if (!(c->ln_eps >= 0.f) || c->flags != 0) return false;
@@ -358,7 +360,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
-  opt_in(reinterpret_cast<const void*>(&modulation_kernel), mod_smem_bytes(cfg->cond_dim));
+  opt_in(reinterpret_cast<const void*>(&modulation_kernel), mod_smem_bytes(kMaxCondDim));  // same for every context
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
   if (e != cudaSuccess) { delete[] ctx->blocks; delete ctx; return DIT_ERR_CUDA; }
   *out = ctx;
@@ -558,3 +560,71 @@ const char* dit_status_string(dit_status s) {
 const char* dit_last_error(const dit_ctx* ctx) { return ctx ? ctx->err : ""; }
 
 }  // extern "C"
+
+// =============================================================================================== no-allocation entry point
+// adaLN modulation vectors without a context, a workspace or any allocation.  The context path keeps
+// the fp32 copy of the modulation bias in the caller's workspace; here that scratch is a fixed
+// array inside the library image, so the call works for hosts that must not allocate device
+// memory.  See include/dit.h for the contract.
+namespace {
+
+constexpr int kNoAllocMaxHidden = 4096;                       // same bound as dit_config.hidden
+constexpr int kNoAllocMaxCond = kMaxCondDim;
+constexpr int kNoAllocScratchFloats = 6 * kNoAllocMaxHidden;  // 96 KiB per GPU that loads the library
+constexpr int kNoAllocMaxDevices = 64;
+
+static __device__ __align__(256) float g_noalloc_bias_scratch[kNoAllocScratchFloats];
+
+// In host code the array's name is only a handle for the runtime; the device address is looked up
+// once per device (with that device current) and cached.
+std::mutex g_noalloc_mutex;
+float* g_noalloc_scratch_ptr[kNoAllocMaxDevices] = {};
+
+cudaError_t noalloc_scratch_for_current_device(float** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_scratch_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_bias_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(&modulation_kernel),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(mod_smem_bytes(kNoAllocMaxCond)));
+    if (e != cudaSuccess) return e;
+    g_noalloc_scratch_ptr[dev] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_scratch_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" dit_status dit_modulation_noalloc(const void* cond, const void* w_ada, const void* b_ada,
+                                             int32_t n_requests, int32_t cond_dim, int32_t hidden, float* mod_out,
+                                             void* stream) {
+  if (n_requests < 0) return DIT_ERR_INVALID_ARG;
+  if (n_requests == 0) return DIT_OK;
+  if (!cond || !w_ada || !mod_out) return DIT_ERR_INVALID_ARG;
+  if (hidden < 64 || hidden % 64 || cond_dim < 1) return DIT_ERR_SHAPE;
+  if (hidden > kNoAllocMaxHidden || cond_dim > kNoAllocMaxCond || n_requests > DIT_MAX_REQUESTS) return DIT_ERR_CAPACITY;
+  float* scratch = nullptr;
+  if (noalloc_scratch_for_current_device(&scratch) != cudaSuccess) return DIT_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n6 = 6 * hidden;
+  // The scratch still holds the previous call's bias: rewrite all of [0, 6H) (zeros for a NULL bias).
+  bf16_to_f32_kernel<<<(n6 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(b_ada), scratch, n6);
+  if (cudaGetLastError() != cudaSuccess) return DIT_ERR_CUDA;
+  ModParams mp{};
+  mp.cond = static_cast<const __nv_bfloat16*>(cond);
+  mp.w_ada0 = static_cast<const __nv_bfloat16*>(w_ada);
+  mp.b_ada0 = scratch;
+  mp.w_block_stride = 0; mp.b_block_stride = 0;
+  mp.mod = mod_out; mp.R = n_requests; mp.C = cond_dim; mp.N6 = n6; mp.NB = 1;
+  modulation_kernel<<<(n6 + kModCols - 1) / kModCols, kModThreads, mod_smem_bytes(cond_dim), st>>>(mp);
+  if (cudaGetLastError() != cudaSuccess) return DIT_ERR_CUDA;
+  return DIT_OK;
+}
