@@ -1,20 +1,24 @@
 // Variable-length multi-head softmax attention for sm_100a, block-diagonal per request.
 //
-// One CTA owns (request, head, 128 query rows).  Tiles are cut relative to the request's first row,
-// never relative to the packed offset, so a request sees the same tiling whether it runs alone or
-// packed with others.  Q, K and V tiles are TMA boxes cut straight out of the packed [T, 3H] fp16
-// qkv buffer (columns head*d, H + head*d, 2H + head*d); V is consumed as an MN-major B operand, so
-// no transpose is ever materialised.  Rows past the end of the batch are zero-filled by TMA, rows
-// past the end of the request belong to the next request (finite values); both are masked out of
-// the softmax before the row maximum is taken.
+// One CTA owns (request, head, 256 query rows) as two 128-row tiles, each served by its own softmax
+// warpgroup.  Tiles are cut relative to the request's first row, never relative to the packed
+// offset, so a request sees the same tiling whether it runs alone or packed with others.  Q, K and
+// V tiles are TMA boxes cut straight out of the packed [T, 3H] fp16 qkv buffer (columns head*d,
+// H + head*d, 2H + head*d); V is consumed as an MN-major B operand, so no transpose is ever
+// materialised.  Rows past the end of the batch are zero-filled by TMA, rows past the end of the
+// request belong to the next request (finite values); both are masked out of the softmax before the
+// row maximum is taken.
 //
-// Pipeline per KV tile j (online softmax, fp32 statistics):
-//   MMA warp     S_j = Q K_j^T            -> TMEM S[j&1]            (tcgen05.mma, fp32 accumulate)
-//   softmax WG   m_j, alpha_j, P_j = exp2(c*(S_j - m_j)) -> fp16 P[j&1] in shared memory (swizzled)
-//   MMA warp     O_j = P_j V_j            -> TMEM O[j&1]            (fresh, not accumulated)
-//   softmax WG   acc = acc * alpha_j + O_j   (fp32 registers, one thread per query row)
-// S_{j+1} is issued before P_j V_j, so the tensor core works on the next scores while the softmax
-// warps exponentiate the current ones.  Output = acc / l, written as fp16 [T, H].
+// Per KV tile j (128 keys) and query tile i (online softmax, fp32 statistics):
+//   MMA warp      S_i = Q_i K_j^T              -> TMEM S[i]            (SS tcgen05.mma)
+//   softmax WG i  m, alpha, P = exp2(c*(S-m))  -> fp16 P over S[i]'s columns (tcgen05.st)
+//   MMA warp      O_i = P_i V_j                -> TMEM O[i], fresh     (TS tcgen05.mma, A = P in TMEM)
+//   softmax WG i  acc = acc * alpha + O_i         (fp32 registers, one thread per query row)
+// The two warpgroups alternate: while one exponentiates, the tensor core runs the other's P V and
+// next Q K^T.  Output = acc / l, written as fp16 [T, H].
+//
+// Thread layout (384): warpgroup 0 = {warp 0: TMA producer, warp 1: MMA issuer + TMEM owner},
+// warpgroups 1 and 2 = softmax for query tile 0 and 1.  Registers are re-balanced with setmaxnreg.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -33,16 +37,15 @@ template <int D>
 struct AttnCfg {
   static constexpr int NP = D / 64;              // 64-column panels per head slice
   static constexpr int PANEL = 128 * 128;        // bytes of one [128 rows x 64 fp16] swizzled panel
-  static constexpr int Q_BYTES = NP * PANEL;
-  static constexpr int KV_BYTES = NP * PANEL;
-  static constexpr int P_BYTES = 2 * PANEL;      // 128 rows x 128 keys fp16
-  static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + Q_BYTES;
-  static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;
-  static constexpr int OFF_P = OFF_V + 2 * KV_BYTES;
-  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
+  static constexpr int TILE_BYTES = NP * PANEL;  // one 128-row Q, K or V tile
+  static constexpr int KV_STAGES = 2;
+  static constexpr int OFF_Q = 0;                                    // two query tiles
+  static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
+  static constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_V + KV_STAGES * TILE_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
-  static constexpr int THREADS = 192;
+  static constexpr int THREADS = 384;
+  static constexpr int Q_ROWS = 256;             // query rows per CTA
 };
 
 __device__ __forceinline__ float exp2_approx(float x) {
@@ -67,27 +70,28 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   auto k_empty = [&](int s) { return bar0 + 8u * (3 + s); };
   auto v_full = [&](int s) { return bar0 + 8u * (5 + s); };
   auto v_empty = [&](int s) { return bar0 + 8u * (7 + s); };
-  auto s_full = [&](int s) { return bar0 + 8u * (9 + s); };
-  auto p_full = [&](int s) { return bar0 + 8u * (11 + s); };
-  auto o_full = [&](int s) { return bar0 + 8u * (13 + s); };
+  auto s_full = [&](int i) { return bar0 + 8u * (9 + i); };
+  auto p_full = [&](int i) { return bar0 + 8u * (11 + i); };
+  auto o_full = [&](int i) { return bar0 + 8u * (13 + i); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + C::OFF_BAR + 8 * 15);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  // ---- which (request, head, query tile) this CTA owns
+  // ---- which (request, head, 256-row query block) this CTA owns
   const int head = blockIdx.x % p.n_heads;
-  int qt = blockIdx.x / p.n_heads;
+  int qb = blockIdx.x / p.n_heads;
   int row_begin = 0, len = 0;
   for (int i = 0; i < seq.n; ++i) {
     const int r = seq.order[i];
     const int l = seq.cu[r + 1] - seq.cu[r];
-    const int nt = (l + 127) >> 7;
-    if (qt < nt) { row_begin = seq.cu[r]; len = l; break; }
-    qt -= nt;
+    const int nb = (l + C::Q_ROWS - 1) / C::Q_ROWS;
+    if (qb < nb) { row_begin = seq.cu[r]; len = l; break; }
+    qb -= nb;
   }
-  const int q_row0 = row_begin + qt * 128;
+  const int q_row0 = row_begin + qb * C::Q_ROWS;
   const int nkv = (len + 127) >> 7;
+  const bool tile1_valid = qb * C::Q_ROWS + 128 < len;     // second query tile has at least one row
   const int xq = head * D, xk = p.H + head * D, xv = 2 * p.H + head * D;
 
   if (threadIdx.x == 0) {
@@ -106,184 +110,179 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // TMEM columns: S[0] 0..127, S[1] 128..255, O[0] 256.., O[1] 384..
+  // TMEM columns: S[0] 0..127, S[1] 128..255 (P[i] overwrites the first 64 columns of S[i]),
+  // O[0] 256.., O[1] 384..
   const uint32_t tS = tmem_base, tO = tmem_base + 256;
 
-  if (len == 0) goto done;   // grid padding (cannot happen with an exact grid)
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
-      for (int pn = 0; pn < C::NP; ++pn)
-        tma_load_2d(base + C::OFF_Q + pn * C::PANEL, &tmQKV, xq + pn * 64, q_row0, q_full);
+  if (warp < 4) {
+    DIT_SETMAXNREG_DEC(40);
+    if (len == 0) goto done;   // grid padding (cannot happen with an exact grid)
+    if (warp == 0 && lane == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      mbar_arrive_expect_tx(q_full, 2 * C::TILE_BYTES);
+      for (int i = 0; i < 2; ++i)
+        for (int pn = 0; pn < C::NP; ++pn)
+          tma_load_2d(base + C::OFF_Q + i * C::TILE_BYTES + pn * C::PANEL, &tmQKV, xq + pn * 64, q_row0 + i * 128, q_full);
       for (int j = 0; j < nkv; ++j) {
-        const int s = j & 1; const uint32_t ph = (j >> 1) & 1u;
+        const int s = j % C::KV_STAGES; const uint32_t ph = (j / C::KV_STAGES) & 1u;
         const int y = row_begin + j * 128;
         if (!mbar_wait(k_empty(s), ph ^ 1u, abort_flag)) goto done;
-        mbar_arrive_expect_tx(k_full(s), C::KV_BYTES);
+        mbar_arrive_expect_tx(k_full(s), C::TILE_BYTES);
         for (int pn = 0; pn < C::NP; ++pn)
-          tma_load_2d(base + C::OFF_K + s * C::KV_BYTES + pn * C::PANEL, &tmQKV, xk + pn * 64, y, k_full(s));
+          tma_load_2d(base + C::OFF_K + s * C::TILE_BYTES + pn * C::PANEL, &tmQKV, xk + pn * 64, y, k_full(s));
         if (!mbar_wait(v_empty(s), ph ^ 1u, abort_flag)) goto done;
-        mbar_arrive_expect_tx(v_full(s), C::KV_BYTES);
+        mbar_arrive_expect_tx(v_full(s), C::TILE_BYTES);
         for (int pn = 0; pn < C::NP; ++pn)
-          tma_load_2d(base + C::OFF_V + s * C::KV_BYTES + pn * C::PANEL, &tmQKV, xv + pn * 64, y, v_full(s));
+          tma_load_2d(base + C::OFF_V + s * C::TILE_BYTES + pn * C::PANEL, &tmQKV, xv + pn * 64, y, v_full(s));
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    } else if (warp == 1 && lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer
       constexpr uint32_t idesc_s = idesc_f16(128, 128, false);
       constexpr uint32_t idesc_pv = idesc_f16(128, D, true);
-      bool ok = true;
-      auto issue_s = [&](int j) {
-        const int s = j & 1;
-        if (!mbar_wait(k_full(s), (j >> 1) & 1u, abort_flag)) { ok = false; return; }
-        tc_fence_after();
-        const uint32_t qa = base + C::OFF_Q, ka = base + C::OFF_K + s * C::KV_BYTES;
+      const int ntile = tile1_valid ? 2 : 1;
+      // S_i(j) = Q_i K_j^T for both query tiles; K stage is released after the last of them
+      auto issue_s = [&](int j, int i) {
+        const int s = j % C::KV_STAGES;
+        const uint32_t qa = base + C::OFF_Q + i * C::TILE_BYTES, ka = base + C::OFF_K + s * C::TILE_BYTES;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * C::PANEL + (kk & 3) * 32;
-          umma_f16(tS + s * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
+          umma_f16(tS + i * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
                    idesc_s, kk != 0);
         }
-        umma_commit(k_empty(s));
-        umma_commit(s_full(s));
+        if (i == ntile - 1) umma_commit(k_empty(s));
+        umma_commit(s_full(i));
       };
       if (!mbar_wait(q_full, 0, abort_flag)) goto done;
-      issue_s(0);
-      if (nkv > 1 && ok) issue_s(1);
-      for (int j = 0; j < nkv && ok; ++j) {
-        const int s = j & 1; const uint32_t ph = (j >> 1) & 1u;
-        if (!mbar_wait(p_full(s), ph, abort_flag)) goto done;
-        if (!mbar_wait(v_full(s), ph, abort_flag)) goto done;
-        tc_fence_after();
-        const uint32_t pa = base + C::OFF_P + s * C::P_BYTES, va = base + C::OFF_V + s * C::KV_BYTES;
+      if (!mbar_wait(k_full(0), 0, abort_flag)) goto done;
+      tc_fence_after();
+      for (int i = 0; i < ntile; ++i) issue_s(0, i);
+      for (int j = 0; j < nkv; ++j) {
+        const int s = j % C::KV_STAGES; const uint32_t ph = (j / C::KV_STAGES) & 1u;
+        for (int i = 0; i < ntile; ++i) {
+          if (!mbar_wait(p_full(i), j & 1u, abort_flag)) goto done;
+          if (i == 0) {
+            if (!mbar_wait(v_full(s), ph, abort_flag)) goto done;
+            if (j + 1 < nkv && !mbar_wait(k_full((j + 1) % C::KV_STAGES), ((j + 1) / C::KV_STAGES) & 1u, abort_flag)) goto done;
+          }
+          tc_fence_after();
+          const uint32_t va = base + C::OFF_V + s * C::TILE_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {       // 16 keys per MMA
-          const uint64_t adesc = smem_desc_sw128(pa + (kk >> 2) * C::PANEL + (kk & 3) * 32, 16, 1024);
-          // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns
-          // live one panel further (leading byte offset).
-          const uint64_t bdesc = smem_desc_sw128(va + kk * 2048, C::PANEL, 1024);
-          umma_f16(tO + s * 128, adesc, bdesc, idesc_pv, kk != 0);
+          for (int kk = 0; kk < 8; ++kk) {       // 16 keys per MMA: 8 TMEM columns of packed fp16 P
+            // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns
+            // live one panel further (leading byte offset).
+            const uint64_t bdesc = smem_desc_sw128(va + kk * 2048, C::PANEL, 1024);
+            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, bdesc, idesc_pv, kk != 0);
+          }
+          if (i == ntile - 1) umma_commit(v_empty(s));
+          umma_commit(o_full(i));
+          // the next scores of this tile go over P_i: the tensor pipe runs them after the P V above
+          if (j + 1 < nkv) issue_s(j + 1, i);
         }
-        umma_commit(v_empty(s));
-        umma_commit(o_full(s));
-        if (j + 2 < nkv) issue_s(j + 2);
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax + accumulate (4 warps)
+    // ------------------------------------------------------------------ softmax + accumulate (2 warpgroups)
+    DIT_SETMAXNREG_INC(232);
+    const int tile = (warp >> 2) - 1;                            // query tile of this warpgroup
     const int quarter = warp & 3;
     const int prow = quarter * 32 + lane;                        // query row inside the tile
+    if (len == 0 || (tile == 1 && !tile1_valid)) goto done;
     const uint32_t lane_sel = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t tSi = tS + tile * 128 + lane_sel, tOi = tO + tile * 128 + lane_sel;
     const float c = p.scale_log2;
-    float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
-    float acc[D];
+    const float2 c2 = make_float2(c, c);
+    float m = -INFINITY, l = 0.f;
+    float2 acc[D / 2];
 #pragma unroll
-    for (int i = 0; i < D; ++i) acc[i] = 0.f;
+    for (int i = 0; i < D / 2; ++i) acc[i] = make_float2(0.f, 0.f);
 
     for (int j = 0; j < nkv; ++j) {
-      const int s = j & 1; const uint32_t ph = (j >> 1) & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full(s), ph, abort_flag))) goto done;
+      const uint32_t ph = j & 1u;
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full(tile), ph, abort_flag))) goto done;
       tc_fence_after();
       const int valid = len - j * 128;                           // keys of this tile inside the request
       // pass 1: row maximum
-      float mx = m;
+      float mx0 = m, mx1 = -INFINITY;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t r[32];
         __syncwarp();
-        tmem_ld32(tS + lane_sel + s * 128 + ch * 32, r);
+        tmem_ld32(tSi + ch * 32, r);
         tmem_ld_wait();
         if (valid >= ch * 32 + 32) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+          for (int i = 0; i < 32; i += 4) {
+            mx0 = fmax3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            mx1 = fmax3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
-            if (ch * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
+            if (ch * 32 + i < valid) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
         }
       }
+      const float mx = fmaxf(mx0, mx1);
       const float alpha = exp2_approx((m - mx) * c);             // m = -inf on the first tile -> 0
       const float neg_mc = -mx * c;
-      // pass 2: P = exp2(c*s - c*m), row sum, fp16 P into swizzled shared memory
-      float rowsum = 0.f;
-      const uint32_t p_row = base + C::OFF_P + s * C::P_BYTES + prow * 128;
+      const float2 nm2 = make_float2(neg_mc, neg_mc);
+      // pass 2: P = exp2(c*s - c*m) as fp16 over the columns S occupied, row sum in fp32
+      float2 rs0 = make_float2(0.f, 0.f), rs1 = make_float2(0.f, 0.f);
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t r[32];
         __syncwarp();
-        tmem_ld32(tS + lane_sel + s * 128 + ch * 32, r);
+        tmem_ld32(tSi + ch * 32, r);
         tmem_ld_wait();
         uint32_t w[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float e0 = exp2_approx(fmaf(__uint_as_float(r[i]), c, neg_mc));
-          float e1 = exp2_approx(fmaf(__uint_as_float(r[i + 1]), c, neg_mc));
-          if (ch * 32 + i >= valid) e0 = 0.f;
-          if (ch * 32 + i + 1 >= valid) e1 = 0.f;
-          rowsum += e0 + e1;
-          const __half2 hh = __floats2half2_rn(e0, e1);
+          const float2 x = ffma2(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), c2, nm2);
+          float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
+          if (ch * 32 + i >= valid) e.x = 0.f;
+          if (ch * 32 + i + 1 >= valid) e.y = 0.f;
+          if (i & 2) rs1 = fadd2(rs1, e); else rs0 = fadd2(rs0, e);
+          const __half2 hh = __floats2half2_rn(e.x, e.y);
           w[i >> 1] = *reinterpret_cast<const uint32_t*>(&hh);
         }
-        const uint32_t panel = p_row + (ch >> 1) * C::PANEL;
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const uint32_t chunk = static_cast<uint32_t>(((ch & 1) * 4 + v) ^ (prow & 7));
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(panel + chunk * 16), "r"(w[4 * v]),
-                       "r"(w[4 * v + 1]), "r"(w[4 * v + 2]), "r"(w[4 * v + 3]) : "memory");
-        }
+        tmem_st16(tSi + ch * 16, w);
       }
-      fence_proxy_async_smem();     // make this thread's P writes visible to the tensor core
-      tc_fence_before();            // and order its TMEM reads of S before the next S MMA
-      mbar_arrive(p_full(s));
-      l = l * alpha + rowsum;
-      // fold in the previous tile's P V product
-      if (j > 0) {
-        const int sp = (j - 1) & 1; const uint32_t php = ((j - 1) >> 1) & 1u;
-        if (!__all_sync(0xffffffffu, mbar_wait(o_full(sp), php, abort_flag))) goto done;
-        tc_fence_after();
-#pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
-          uint32_t r[32];
-          __syncwarp();
-          tmem_ld32(tO + lane_sel + sp * 128 + ch * 32, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) acc[ch * 32 + i] = fmaf(acc[ch * 32 + i], alpha_prev, __uint_as_float(r[i]));
-        }
-      }
-      alpha_prev = alpha;
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(p_full(tile));
+      l = l * alpha + ((rs0.x + rs0.y) + (rs1.x + rs1.y));
       m = mx;
-    }
-    {
-      const int sp = (nkv - 1) & 1; const uint32_t php = ((nkv - 1) >> 1) & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(o_full(sp), php, abort_flag))) goto done;
+      // fold in this tile's P V product
+      if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), ph, abort_flag))) goto done;
       tc_fence_after();
-      const float inv = 1.0f / l;
-      const bool row_ok = qt * 128 + prow < len;
-      __half* dst = p.out + static_cast<size_t>(q_row0 + prow) * p.H + head * D;
+      const float2 a2 = make_float2(alpha, alpha);
 #pragma unroll
       for (int ch = 0; ch < D / 32; ++ch) {
         uint32_t r[32];
         __syncwarp();
-        tmem_ld32(tO + lane_sel + sp * 128 + ch * 32, r);
+        tmem_ld32(tOi + ch * 32, r);
         tmem_ld_wait();
-        if (row_ok) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint32_t w[4];
+        for (int i = 0; i < 32; i += 2)
+          acc[ch * 16 + (i >> 1)] = ffma2(acc[ch * 16 + (i >> 1)], a2, make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+      }
+      tc_fence_before();   // orders these TMEM reads before the arrival that lets the next P V overwrite O
+    }
+    {
+      const float inv = 1.0f / l;
+      const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
+      if (row_in_req < len) {
+        __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.H + head * D;
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const int i = 8 * v + 2 * h;
-              const float a = fmaf(acc[ch * 32 + i], alpha_prev, __uint_as_float(r[i])) * inv;
-              const float b = fmaf(acc[ch * 32 + i + 1], alpha_prev, __uint_as_float(r[i + 1])) * inv;
-              const __half2 hh = __floats2half2_rn(a, b);
-              w[h] = *reinterpret_cast<const uint32_t*>(&hh);
-            }
-            *(reinterpret_cast<uint4*>(dst + ch * 32) + v) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int v = 0; v < D / 8; ++v) {
+          uint32_t w[4];
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            const float2 a = acc[4 * v + h];
+            const __half2 hh = __floats2half2_rn(a.x * inv, a.y * inv);
+            w[h] = *reinterpret_cast<const uint32_t*>(&hh);
           }
+          *(reinterpret_cast<uint4*>(dst) + v) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }

@@ -155,9 +155,9 @@ cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtens
 
 template <int D>
 cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, const SeqInfo& seq, cudaStream_t st) {
-  int qtiles = 0;
-  for (int r = 0; r < seq.n; ++r) qtiles += (seq.cu[r + 1] - seq.cu[r] + 127) / 128;
-  attention_tcgen05_kernel<D><<<qtiles * p.n_heads, AttnCfg<D>::THREADS, AttnCfg<D>::SMEM_BYTES, st>>>(tmQKV, p, seq);
+  int qblocks = 0;
+  for (int r = 0; r < seq.n; ++r) qblocks += (seq.cu[r + 1] - seq.cu[r] + AttnCfg<D>::Q_ROWS - 1) / AttnCfg<D>::Q_ROWS;
+  attention_tcgen05_kernel<D><<<qblocks * p.n_heads, AttnCfg<D>::THREADS, AttnCfg<D>::SMEM_BYTES, st>>>(tmQKV, p, seq);
   return cudaGetLastError();
 }
 
