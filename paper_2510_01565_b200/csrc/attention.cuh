@@ -12,8 +12,10 @@
 // Per KV tile j (128 keys) and query tile i (online softmax, fp32 statistics):
 //   MMA warp      S_i = Q_i K_j^T              -> TMEM S[i]            (SS tcgen05.mma)
 //   softmax WG i  m, alpha, P = exp2(c*(S-m))  -> fp16 P over S[i]'s columns (tcgen05.st)
-//   MMA warp      O_i = P_i V_j                -> TMEM O[i], fresh     (TS tcgen05.mma, A = P in TMEM)
-//   softmax WG i  acc = acc * alpha + O_i         (fp32 registers, one thread per query row)
+//   MMA warp      O_i += P_i V_j               -> TMEM O[i]            (TS tcgen05.mma, A = P in TMEM)
+// O is rescaled in TMEM only when a row maximum has grown by more than 2^8 since the reference was
+// set (rare after the first tiles); P is bounded by 2^8, and O and l share the reference, so the
+// normalised result is the same.
 // The two warpgroups alternate: while one exponentiates, the tensor core runs the other's P V and
 // next Q K^T.  Output = acc / l, written as fp16 [T, H].
 //
@@ -172,7 +174,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
             // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns
             // live one panel further (leading byte offset).
             const uint64_t bdesc = smem_desc_sw128(va + kk * 2048, C::PANEL, 1024);
-            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, bdesc, idesc_pv, kk != 0);
+            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, bdesc, idesc_pv, (j | kk) != 0);
           }
           if (i == ntile - 1) umma_commit(v_empty(s));
           umma_commit(o_full(i));
@@ -192,55 +194,71 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
     const uint32_t tSi = tS + tile * 128 + lane_sel, tOi = tO + tile * 128 + lane_sel;
     const float c = p.scale_log2;
     const float2 c2 = make_float2(c, c);
-    float m = -INFINITY, l = 0.f;
-    float2 acc[D / 2];
-#pragma unroll
-    for (int i = 0; i < D / 2; ++i) acc[i] = make_float2(0.f, 0.f);
+    // Running reference maximum m_ref (scores are exponentiated relative to it) and row sum l.
+    // O accumulates in TMEM; it is rescaled only when a row's maximum has grown by more than
+    // kRescaleLog2 in the exponent, so P stays <= 2^kRescaleLog2 and the result is unchanged
+    // (both O and l carry the same reference).
+    constexpr float kRescaleLog2 = 8.0f;
+    float m_ref = -INFINITY, l = 0.f;
 
     for (int j = 0; j < nkv; ++j) {
       const uint32_t ph = j & 1u;
       if (!__all_sync(0xffffffffu, mbar_wait(s_full(tile), ph, abort_flag))) goto done;
       tc_fence_after();
       const int valid = len - j * 128;                           // keys of this tile inside the request
-      // pass 1: row maximum
-      float mx0 = m, mx1 = -INFINITY;
+      uint32_t sv[128];                                          // this row's 128 scores
+      __syncwarp();
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) tmem_ld32p(tSi + ch * 32, sv + ch * 32);
+      tmem_ld_wait();
+      if (valid < 128) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i >= valid) sv[i] = 0xff800000u;                   // -inf: drops out of max and sum
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 8) {
+        mx0 = fmax3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+        mx1 = fmax3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+        mx2 = fmax3(mx2, __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
+        mx3 = fmax3(mx3, __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      if (j == 0) {
+        m_ref = mx;
+      } else {
+        const bool grow = (mx - m_ref) * c > kRescaleLog2;
+        if (__any_sync(0xffffffffu, grow)) {
+          // rare: rescale this warp's rows of O (rows that did not grow are multiplied by 1)
+          if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), (j - 1) & 1u, abort_flag))) goto done;
+          tc_fence_after();
+          const float alpha = grow ? exp2_approx((m_ref - mx) * c) : 1.0f;
+          if (grow) { m_ref = mx; l *= alpha; }
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        __syncwarp();
-        tmem_ld32(tSi + ch * 32, r);
-        tmem_ld_wait();
-        if (valid >= ch * 32 + 32) {
+          for (int ch = 0; ch < D / 32; ++ch) {
+            uint32_t r[32];
+            __syncwarp();
+            tmem_ld32(tOi + ch * 32, r);
+            tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            mx0 = fmax3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-            mx1 = fmax3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st32(tOi + ch * 32, r);
           }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (ch * 32 + i < valid) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+          tmem_st_wait();
         }
       }
-      const float mx = fmaxf(mx0, mx1);
-      const float alpha = exp2_approx((m - mx) * c);             // m = -inf on the first tile -> 0
-      const float neg_mc = -mx * c;
+      const float neg_mc = -m_ref * c;
       const float2 nm2 = make_float2(neg_mc, neg_mc);
-      // pass 2: P = exp2(c*s - c*m) as fp16 over the columns S occupied, row sum in fp32
+      // P = exp2(c*s - c*m_ref) as fp16 over the columns S occupied, row sum in fp32
       float2 rs0 = make_float2(0.f, 0.f), rs1 = make_float2(0.f, 0.f);
-#pragma unroll 1
+#pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        __syncwarp();
-        tmem_ld32(tSi + ch * 32, r);
-        tmem_ld_wait();
         uint32_t w[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          const float2 x = ffma2(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), c2, nm2);
-          float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
-          if (ch * 32 + i >= valid) e.x = 0.f;
-          if (ch * 32 + i + 1 >= valid) e.y = 0.f;
+          const float2 x = ffma2(make_float2(__uint_as_float(sv[ch * 32 + i]), __uint_as_float(sv[ch * 32 + i + 1])), c2, nm2);
+          const float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
           if (i & 2) rs1 = fadd2(rs1, e); else rs0 = fadd2(rs0, e);
           const __half2 hh = __floats2half2_rn(e.x, e.y);
           w[i >> 1] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -250,39 +268,33 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(p_full(tile));
-      l = l * alpha + ((rs0.x + rs0.y) + (rs1.x + rs1.y));
-      m = mx;
-      // fold in this tile's P V product
-      if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), ph, abort_flag))) goto done;
+      l += (rs0.x + rs0.y) + (rs1.x + rs1.y);
+    }
+    {
+      // the last P V product has landed: normalise and write this row
+      if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), (nkv - 1) & 1u, abort_flag))) goto done;
       tc_fence_after();
-      const float2 a2 = make_float2(alpha, alpha);
-#pragma unroll
+      const float inv = 1.0f / l;
+      const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
+      __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.H + head * D;
+#pragma unroll 1
       for (int ch = 0; ch < D / 32; ++ch) {
         uint32_t r[32];
         __syncwarp();
         tmem_ld32(tOi + ch * 32, r);
         tmem_ld_wait();
+        if (row_in_req < len) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 2)
-          acc[ch * 16 + (i >> 1)] = ffma2(acc[ch * 16 + (i >> 1)], a2, make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
-      }
-      tc_fence_before();   // orders these TMEM reads before the arrival that lets the next P V overwrite O
-    }
-    {
-      const float inv = 1.0f / l;
-      const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
-      if (row_in_req < len) {
-        __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.H + head * D;
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
 #pragma unroll
-        for (int v = 0; v < D / 8; ++v) {
-          uint32_t w[4];
-#pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            const float2 a = acc[4 * v + h];
-            const __half2 hh = __floats2half2_rn(a.x * inv, a.y * inv);
-            w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+            for (int h = 0; h < 4; ++h) {
+              const int i = 8 * v + 2 * h;
+              const __half2 hh = __floats2half2_rn(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+              w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+            }
+            *(reinterpret_cast<uint4*>(dst + ch * 32) + v) = make_uint4(w[0], w[1], w[2], w[3]);
           }
-          *(reinterpret_cast<uint4*>(dst) + v) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }
