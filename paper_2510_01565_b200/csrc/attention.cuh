@@ -117,7 +117,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   const uint32_t tS = tmem_base, tO = tmem_base + 256;
 
   if (warp < 4) {
-    DIT_SETMAXNREG_DEC(40);
+    DIT_SETMAXNREG_DEC(96);
     if (len == 0) goto done;   // grid padding (cannot happen with an exact grid)
     if (warp == 0 && lane == 0) {
       // ------------------------------------------------------------------ TMA producer
@@ -142,15 +142,22 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       constexpr uint32_t idesc_s = idesc_f16(128, 128, false);
       constexpr uint32_t idesc_pv = idesc_f16(128, D, true);
       const int ntile = tile1_valid ? 2 : 1;
-      // S_i(j) = Q_i K_j^T for both query tiles; K stage is released after the last of them
+      // Descriptors are built once; inside the loops only constant offsets are added (>> 4 units).
+      static_assert(C::KV_STAGES == 2, "descriptor selection below assumes two stages");
+      const uint64_t qdesc0 = smem_desc_sw128(base + C::OFF_Q, 16, 1024);
+      const uint64_t kdesc0 = smem_desc_sw128(base + C::OFF_K, 16, 1024);
+      // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns live
+      // one panel further (leading byte offset).
+      const uint64_t vdesc0 = smem_desc_sw128(base + C::OFF_V, C::PANEL, 1024);
+      constexpr uint32_t kTileStep = C::TILE_BYTES >> 4;
+      // S_i(j) = Q_i K_j^T; the K stage is released after the last query tile has used it
       auto issue_s = [&](int j, int i) {
         const int s = j % C::KV_STAGES;
-        const uint32_t qa = base + C::OFF_Q + i * C::TILE_BYTES, ka = base + C::OFF_K + s * C::TILE_BYTES;
+        const uint64_t qd = qdesc0 + i * kTileStep, kd = kdesc0 + s * kTileStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * C::PANEL + (kk & 3) * 32;
-          umma_f16(tS + i * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
-                   idesc_s, kk != 0);
+          const uint32_t off = ((kk >> 2) * C::PANEL + (kk & 3) * 32) >> 4;
+          umma_f16(tS + i * 128, qd + off, kd + off, idesc_s, kk != 0);
         }
         if (i == ntile - 1) umma_commit(k_empty(s));
         umma_commit(s_full(i));
@@ -161,21 +168,16 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       for (int i = 0; i < ntile; ++i) issue_s(0, i);
       for (int j = 0; j < nkv; ++j) {
         const int s = j % C::KV_STAGES; const uint32_t ph = (j / C::KV_STAGES) & 1u;
+        // operands of this round were requested a whole round ago: check them off the critical path
+        if (!mbar_wait(v_full(s), ph, abort_flag)) goto done;
+        if (j + 1 < nkv && !mbar_wait(k_full((j + 1) % C::KV_STAGES), ((j + 1) / C::KV_STAGES) & 1u, abort_flag)) goto done;
         for (int i = 0; i < ntile; ++i) {
           if (!mbar_wait(p_full(i), j & 1u, abort_flag)) goto done;
-          if (i == 0) {
-            if (!mbar_wait(v_full(s), ph, abort_flag)) goto done;
-            if (j + 1 < nkv && !mbar_wait(k_full((j + 1) % C::KV_STAGES), ((j + 1) / C::KV_STAGES) & 1u, abort_flag)) goto done;
-          }
           tc_fence_after();
-          const uint32_t va = base + C::OFF_V + s * C::TILE_BYTES;
+          const uint64_t vd = vdesc0 + s * kTileStep;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {       // 16 keys per MMA: 8 TMEM columns of packed fp16 P
-            // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns
-            // live one panel further (leading byte offset).
-            const uint64_t bdesc = smem_desc_sw128(va + kk * 2048, C::PANEL, 1024);
-            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, bdesc, idesc_pv, (j | kk) != 0);
-          }
+          for (int kk = 0; kk < 8; ++kk)         // 16 keys per MMA: 8 TMEM columns of packed fp16 P
+            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, vd + kk * (2048 >> 4), idesc_pv, (j | kk) != 0);
           if (i == ntile - 1) umma_commit(v_empty(s));
           umma_commit(o_full(i));
           // the next scores of this tile go over P_i: the tensor pipe runs them after the P V above
@@ -185,7 +187,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
     }
   } else {
     // ------------------------------------------------------------------ softmax + accumulate (2 warpgroups)
-    DIT_SETMAXNREG_INC(232);
+    DIT_SETMAXNREG_INC(200);
     const int tile = (warp >> 2) - 1;                            // query tile of this warpgroup
     const int quarter = warp & 3;
     const int prow = quarter * 32 + lane;                        // query row inside the tile

@@ -161,6 +161,17 @@ cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, cons
   return cudaGetLastError();
 }
 
+// LayerNorm + modulate launch: picks the register-resident row width (float4 per lane) for H.
+template <bool kFromBf16>
+cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
+                      long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st) {
+  const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
+  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
+  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
+  else ln_modulate_kernel<kFromBf16, 32><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
+  return cudaGetLastError();
+}
+
 size_t mod_smem_bytes(int C) { return (static_cast<size_t>(kModReqGroup) * C + 8 * kModReqGroup * kModCols) * sizeof(float); }
 
 dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
@@ -225,18 +236,14 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }));
   }
 
-  const int ln_grid = (T + kLnWarps - 1) / kLnWarps;
   for (int b = 0; b < n_blocks; ++b) {
     const BlockState& bs = ctx->blocks[b];
     const uint8_t* wb = ctx->block_base(b);
     const float* modb = mod + static_cast<size_t>(b) * 6 * H;   // request 0; request r at + r * req_stride
     // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      if (b == 0)
-        ln_modulate_kernel<true><<<ln_grid, kLnWarps * 32, 0, st>>>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
-      else
-        ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq);
-      return cudaGetLastError();
+      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st)
+                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st);
     }));
     // QKV projection
     GemmParams g{};
@@ -262,8 +269,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st); }));
     // LN2 + modulate
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      ln_modulate_kernel<false><<<ln_grid, kLnWarps * 32, 0, st>>>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq);
-      return cudaGetLastError();
+      return launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st);
     }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};

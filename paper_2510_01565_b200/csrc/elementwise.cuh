@@ -97,14 +97,15 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 // ------------------------------------------------------------------------------------------------
 // LayerNorm (over H, biased variance, eps inside the root, no affine) + adaLN modulate:
 //   h[row, :] = (x - mean) * rstd * (1 + scale[req]) + shift[req]        -> fp16
-// One warp per row, the row held in registers (H <= 4096), two-pass statistics, fixed shuffle order.
+// One warp per row, the row held in registers (kVec float4 per lane: H <= 128 * kVec), two-pass
+// statistics, fixed shuffle order.  Small CTAs (4 rows) and a register budget that lets several CTAs
+// share an SM keep enough loads in flight to cover HBM latency.
 // kFromBf16 = true reads the packed bf16 tokens (first block) and also writes the fp32 residual stream.
 // ------------------------------------------------------------------------------------------------
-constexpr int kLnWarps = 8;
-constexpr int kLnMaxVec = 32;   // float4 per lane: H <= 32 * 32 * 4 = 4096
+constexpr int kLnWarps = 4;
 
-template <bool kFromBf16>
-__global__ void __launch_bounds__(kLnWarps * 32)
+template <bool kFromBf16, int kLnMaxVec>
+__global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVec <= 24 ? 4 : 3)))
 ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
                    const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                    int T, int H, float eps, const __grid_constant__ SeqInfo seq) {

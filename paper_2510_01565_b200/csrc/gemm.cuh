@@ -37,7 +37,8 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_STAGE_FLOATS = 32 * 33;          // per epilogue warp: 32 rows x 32 columns, padded
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * EPI_STAGE_FLOATS * 4;
 }  // namespace gemm_cfg
 
 __device__ __forceinline__ float gelu_tanh_f32(float z) {
@@ -66,6 +67,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* epi_stage = reinterpret_cast<float*>(aligned + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_m = (p.M + BM - 1) / BM, num_n = (p.N + BN - 1) / BN;
@@ -135,8 +137,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
-      const float* gate_row = nullptr;
-      if (EPI == kEpiGateResidF32 && row_ok) gate_row = p.gate + find_request(seq, row) * p.gate_stride;
+      // gated-residual epilogue: request of this lane's row, and whether the warp's rows share it
+      int my_req = -1;
+      if (EPI == kEpiGateResidF32 && row_ok) my_req = find_request(seq, row);
+      const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
+      const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
@@ -147,31 +152,45 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tmem_ld32(t_row + c * 32, r);
         tmem_ld_wait();
         const int col0 = n0 + c * 32;
-        const bool full = (col0 + 32 <= p.N);
-        if (!row_ok || col0 >= p.N) {
-          // nothing to store for this lane / chunk
-        } else if (EPI == kEpiGateResidF32) {
-          const float* res = p.resid + static_cast<size_t>(row) * p.N + col0;
-          float* dst = p.out32 + static_cast<size_t>(row) * p.N + col0;
-          if (full) {
+        if (col0 >= p.N) continue;             // warp-uniform
+        if (EPI == kEpiGateResidF32) {
+          // Transpose through shared memory so that each global access covers whole 128-byte row
+          // segments: lane -> (row it*4 + lane/8, columns (lane%8)*4 .. +3).
+          float* st = epi_stage + (warp - 2) * EPI_STAGE_FLOATS;
 #pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col0) + v);
-              const float4 g = __ldg(reinterpret_cast<const float4*>(gate_row + col0) + v);
-              const float4 x = *(reinterpret_cast<const float4*>(res) + v);
-              float4 o;
-              o.x = x.x + g.x * (__uint_as_float(r[4 * v + 0]) + b.x);
-              o.y = x.y + g.y * (__uint_as_float(r[4 * v + 1]) + b.y);
-              o.z = x.z + g.z * (__uint_as_float(r[4 * v + 2]) + b.z);
-              o.w = x.w + g.w * (__uint_as_float(r[4 * v + 3]) + b.w);
-              *(reinterpret_cast<float4*>(dst) + v) = o;
+          for (int i = 0; i < 32; ++i) st[lane * 33 + i] = __uint_as_float(r[i]);
+          __syncwarp();
+          const int cg = (lane & 7) * 4, col = col0 + cg;   // N is a multiple of 64: the whole chunk is inside
+          {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+            float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(p.gate + req0 * p.gate_stride + col));
+            float4 x[8];
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              const int grow = m0 + quarter * 32 + it * 4 + (lane >> 3);
+              if (grow < p.M) x[it] = *reinterpret_cast<const float4*>(p.resid + static_cast<size_t>(grow) * p.N + col);
             }
-          } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (col0 + i < p.N) dst[i] = res[i] + gate_row[col0 + i] * (__uint_as_float(r[i]) + p.bias[col0 + i]);
+            for (int it = 0; it < 8; ++it) {
+              const int rr = it * 4 + (lane >> 3);
+              const int grow = m0 + quarter * 32 + rr;
+              const int rq = __shfl_sync(0xffffffffu, my_req, rr);
+              if (grow < p.M) {
+                if (!one_req) g = __ldg(reinterpret_cast<const float4*>(p.gate + rq * p.gate_stride + col));
+                const float* a = st + rr * 33 + cg;
+                float4 o;
+                o.x = x[it].x + g.x * (a[0] + b.x);
+                o.y = x[it].y + g.y * (a[1] + b.y);
+                o.z = x[it].z + g.z * (a[2] + b.z);
+                o.w = x[it].w + g.w * (a[3] + b.w);
+                *reinterpret_cast<float4*>(p.out32 + static_cast<size_t>(grow) * p.N + col) = o;
+              }
+            }
           }
-        } else {
+          __syncwarp();                        // staging buffer is reused by the next chunk
+        } else if (row_ok) {
+          const bool full = (col0 + 32 <= p.N);
           __half* dst = p.out16 + static_cast<size_t>(row) * p.N + col0;
           if (full) {
 #pragma unroll

@@ -53,18 +53,21 @@ constexpr uint64_t kWaitLimitNs = 4000000000ull;
 // Bounded wait.  Returns false when `*abort_flag` (shared memory, set by any thread of the CTA
 // that gave up) is raised or the limit ran out; in the latter case it raises the flag itself.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < 2048; ++i)
+  // try_wait suspends the thread in hardware until the phase completes or a short system limit
+  // passes, so this loop is not a hot spin; the timer, the abort flag and the back-off only come
+  // into play for waits far longer than any healthy one.
+  for (int i = 0; i < (1 << 16); ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   while (true) {
-    for (int i = 0; i < 256; ++i)
+    for (int i = 0; i < 1024; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) {
       *abort_flag = 1;
       return false;
     }
-    __nanosleep(128);
+    __nanosleep(64);
   }
 }
 
