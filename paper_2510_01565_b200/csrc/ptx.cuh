@@ -4,6 +4,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#ifndef DIT_MBAR_SUSPEND_NS
+#define DIT_MBAR_SUSPEND_NS 100000u
+#endif
+
 namespace dit {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -41,6 +45,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
+// try_wait with a suspend-time hint (ns): the waiting thread is parked by the hardware instead of
+// re-polling, so it does not take issue slots from the warps that share its scheduler.
+__device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok;
+}
+
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -57,7 +73,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   // passes, so this loop is not a hot spin; the timer, the abort flag and the back-off only come
   // into play for waits far longer than any healthy one.
   for (int i = 0; i < (1 << 16); ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, DIT_MBAR_SUSPEND_NS)) return true;
   const uint64_t t0 = global_ns();
   while (true) {
     for (int i = 0; i < 1024; ++i)
@@ -170,6 +186,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -180,6 +202,9 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // Two fp32 lanes per instruction (sm_100): d = a * b + c, d = a + b.
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+#ifdef DIT_NO_F32X2
+  return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y));
+#endif
   unsigned long long d;
   asm("fma.rn.f32x2 %0, %1, %2, %3;"
       : "=l"(d)
@@ -188,6 +213,9 @@ __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
   return *reinterpret_cast<float2*>(&d);
 }
 __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+#ifdef DIT_NO_F32X2
+  return make_float2(a.x + b.x, a.y + b.y);
+#endif
   unsigned long long d;
   asm("add.rn.f32x2 %0, %1, %2;"
       : "=l"(d)
