@@ -92,6 +92,7 @@ struct dit_ctx {
   uint8_t* ws;
   EncodeTiledFn encode;
   int num_sms;
+  int gemm_pairs;                          // CTA pairs of the GEMM kernel that fit on the device at once
   BlockState* blocks;
   int64_t last_launches;
   int last_T, last_R, last_nb;
@@ -148,8 +149,9 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
 template <int EPI>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                         const SeqInfo& seq, cudaStream_t st) {
-  const int tiles = ((p.M + gemm_cfg::BM - 1) / gemm_cfg::BM) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
-  const int grid = std::min(tiles, ctx->num_sms);
+  // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
+  const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
+  const int grid = 2 * std::min(tiles, ctx->gemm_pairs);
   gemm_tcgen05_kernel<EPI><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, p, seq);
   return cudaGetLastError();
 }
@@ -371,6 +373,17 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel), mod_smem_bytes(kMaxCondDim));  // same for every context
+  if (e == cudaSuccess) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(sms & ~1); lc.blockDim = dim3(gemm_cfg::THREADS); lc.dynamicSmemBytes = gemm_cfg::SMEM_BYTES;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeClusterDimension;
+    at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    lc.attrs = &at; lc.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16>), &lc);
+    ctx->gemm_pairs = std::max(1, std::min(clusters, sms / 2));
+  }
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
   if (e != cudaSuccess) { delete[] ctx->blocks; delete ctx; return DIT_ERR_CUDA; }
   *out = ctx;
@@ -418,10 +431,10 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   DIT_CUDA_TRY(ctx, weight(w->w_fc2, L.w_fc2, F, H));
   DIT_CUDA_TRY(ctx, bias(w->b_fc2, L.b_fc2, H));
 
-  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN) ||
-      !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN) ||
-      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN) ||
-      !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN))
+  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) ||
+      !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) ||
+      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) ||
+      !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;
   return DIT_OK;

@@ -1,12 +1,17 @@
 // Persistent warp-specialised GEMM for sm_100a:  C[M,N] = A[M,K] * Wt[N,K]^T  (+ fused epilogue).
 //
 // A (activations, fp16, row-major [M,K]) and Wt (weights, fp16, row-major [N,K]) are both K-major.
-// TMA brings 128x64 (A) and 256x64 (Wt) tiles with the 128-byte swizzle into a 4-stage shared-memory
-// ring; one thread issues tcgen05.mma (128x256x16, kind::f16, fp32 accumulate) into one of two TMEM
-// accumulators (2 x 256 columns), so that the epilogue of a tile overlaps the main loop of the next.
-// Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue (one TMEM lane
-// quarter each).  Tiles are taken in a fixed order and every output element is accumulated over K in
-// the same order whatever M is: a row's result does not depend on where it sits in the batch.
+// Two CTAs on neighbouring SMs (a cluster of 2) share one 256x256 output tile: each CTA loads its own
+// 128 rows of A and one half (128 rows) of the Wt tile per 64-wide K step (TMA, 128-byte swizzle,
+// 6-stage ring of 32 KB), and one thread of the leader CTA issues tcgen05.mma.cta_group::2
+// (256x256x16, kind::f16, fp32 accumulate).  Each CTA ends up with its 128 rows x 256 columns in one of
+// two TMEM accumulators, so the epilogue of a tile overlaps the main loop of the next.  Compared with
+// one CTA per 128x256 tile this halves the shared-memory and L2 traffic for the weight operand.
+// No TMA multicast is used: both CTAs' loads report their bytes to the leader's barrier, and
+// tcgen05.commit (multicast over the pair) releases stages and publishes accumulators in both CTAs.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer (leader CTA only) and TMEM owner, 2..5 = epilogue (one
+// TMEM lane quarter each).  Tiles are taken in a fixed order and every output element is accumulated
+// over K in the same order whatever M is: a row's result does not depend on where it sits in the batch.
 //
 // Epilogues (the fused parts of the adaLN-Zero block):
 //   kEpiBiasF16      out16 = acc + bias                                   (QKV projection)
@@ -32,9 +37,9 @@ struct GemmParams {
 };
 
 namespace gemm_cfg {
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 6;     // BM: rows per CTA; the pair covers 2*BM x BN
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
+constexpr int B_BYTES = (BN / 2) * BK * 2;                  // this CTA's half of the weight tile
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr int EPI_STAGE_FLOATS = 32 * 33;          // per epilogue warp: 32 rows x 32 columns, padded
@@ -50,7 +55,7 @@ __device__ __forceinline__ float gelu_tanh_f32(float z) {
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(gemm_cfg::THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmParams p, const __grid_constant__ SeqInfo seq) {
   using namespace gemm_cfg;
@@ -59,7 +64,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* aligned = smem_raw + (base - raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
-  // bars: [0,S) full, [S,2S) empty, [2S,2S+2) tmem_full, [2S+2,2S+4) tmem_empty
+  // bars: [0,S) full (used in the leader), [S,2S) empty, [2S,2S+2) tmem_full, [2S+2,2S+4) tmem_empty (leader)
   const uint32_t bar0 = base + STAGES * STAGE_BYTES;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -70,45 +75,50 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   float* epi_stage = reinterpret_cast<float*>(aligned + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_m = (p.M + BM - 1) / BM, num_n = (p.N + BN - 1) / BN;
-  const int num_tiles = num_m * num_n;
+  const uint32_t rank = cluster_ctarank();                    // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int num_m = (p.M + 2 * BM - 1) / (2 * BM), num_n = (p.N + BN - 1) / BN;
+  const int num_tiles = num_m * num_n;                        // 256 x 256 tiles
   const int num_k = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmA); prefetch_tmap(&tmB); }
-  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc_pair(smem_u32(tmem_slot), 512); tmem_relinquish_pair(); }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                                         // both CTAs' barriers exist before any remote arrive
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-        const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+      for (int t = pair; t < num_tiles; t += num_pairs) {
+        const int m0 = (t % num_m) * (2 * BM) + rank * BM;    // this CTA's rows of A
+        const int n0 = (t / num_m) * BN + rank * (BN / 2);    // this CTA's half of the weight tile
         for (int kb = 0; kb < num_k; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) goto done;
-          mbar_arrive_expect_tx(full_bar(stage), STAGE_BYTES);
+          const uint32_t full_leader = map_to_cta(full_bar(stage), 0);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE_BYTES);   // both CTAs' bytes
           const uint32_t sa = base + stage * STAGE_BYTES;
-          tma_load_2d(sa, &tmA, kb * BK, m0, full_bar(stage));
-          tma_load_2d(sa + A_BYTES, &tmB, kb * BK, n0, full_bar(stage));
+          tma_load_2d_pair(sa, &tmA, kb * BK, m0, full_leader);
+          tma_load_2d_pair(sa + A_BYTES, &tmB, kb * BK, n0, full_leader);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_f16(BM, BN, false);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = idesc_f16(2 * BM, BN, false);
       int stage = 0; uint32_t phase = 0; int it = 0;
-      for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+      for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
         const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) goto done;
         tc_fence_after();
@@ -121,20 +131,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint64_t bdesc = smem_desc_sw128(sa + A_BYTES, 16, 1024);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)   // 32 bytes further along K inside the swizzled row
-            umma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-          umma_commit(empty_bar(stage));       // frees the stage once these MMAs have read it
+            umma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        umma_commit(tfull_bar(acc));           // accumulator complete
+        umma_commit_pair(tfull_bar(acc), 3);       // accumulator complete in both CTAs
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps)
     const int quarter = warp & 3;              // TMEM lanes this warp may read: [32*quarter, +32)
     int it = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+    const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
+    for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
       const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
-      const int m0 = (t % num_m) * BM, n0 = (t / num_m) * BN;
+      const int m0 = (t % num_m) * (2 * BM) + rank * BM, n0 = (t / num_m) * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
       // gated-residual epilogue: request of this lane's row, and whether the warp's rows share it
@@ -221,14 +232,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);   // 8 arrivals: 4 warps x 2 CTAs
     }
   }
 
 done:
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+  cluster_sync_all();        // the peer may still signal this CTA's barriers or read its operands until here
+  if (warp == 1) { tc_fence_after(); tmem_dealloc_pair(tmem_base, 512); }
   if (threadIdx.x == 0 && *abort_flag) atomicMax(p.status, kStatusGemmTimeout);
 }
 
