@@ -149,10 +149,14 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
 template <int EPI>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                         const SeqInfo& seq, cudaStream_t st) {
+  // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
+  GemmParams q = p;
+  const long long band_bytes = 2ll * gemm_cfg::BM * p.K * 2;
+  q.band = static_cast<int>(std::max(1ll, std::min<long long>((36ll << 20) / band_bytes, (p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM))));
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);
-  gemm_tcgen05_kernel<EPI><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, p, seq);
+  gemm_tcgen05_kernel<EPI><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, q, seq);
   return cudaGetLastError();
 }
 

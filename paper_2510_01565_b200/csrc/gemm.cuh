@@ -27,6 +27,7 @@ enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32
 
 struct GemmParams {
   int M, N, K;
+  int band;                 // row tiles (of 256 rows) per band of the tile order, >= 1
   const float* bias;        // [N]
   __half* out16;            // [M, N]
   const float* resid;       // [M, N]
@@ -52,6 +53,18 @@ __device__ __forceinline__ float gelu_tanh_f32(float z) {
   float t;
   asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(y));
   return 0.5f * z * (1.0f + t);
+}
+
+// Tile order.  Row tiles are grouped in bands of `band`; inside a band the row index runs fastest and
+// every column tile is visited before the next band starts.  The tiles in flight then share one
+// band of A (sized by the host to stay in L2) while the weight tiles stream past, each read from
+// DRAM once per band.
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int band, int& mb, int& nb) {
+  const int per_band = band * num_n;
+  const int b = t / per_band, r = t - b * per_band;
+  const int rows = min(band, num_m - b * band);               // the last band may be shorter
+  nb = r / rows;
+  mb = b * band + (r - nb * rows);
 }
 
 template <int EPI>
@@ -100,8 +113,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       for (int t = pair; t < num_tiles; t += num_pairs) {
-        const int m0 = (t % num_m) * (2 * BM) + rank * BM;    // this CTA's rows of A
-        const int n0 = (t / num_m) * BN + rank * (BN / 2);    // this CTA's half of the weight tile
+        int mb, nb;
+        tile_coords(t, num_m, num_n, p.band, mb, nb);
+        const int m0 = mb * (2 * BM) + rank * BM;             // this CTA's rows of A
+        const int n0 = nb * BN + rank * (BN / 2);             // this CTA's half of the weight tile
         for (int kb = 0; kb < num_k; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) goto done;
           const uint32_t full_leader = map_to_cta(full_bar(stage), 0);
@@ -145,7 +160,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
     for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
       const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
-      const int m0 = (t % num_m) * (2 * BM) + rank * BM, n0 = (t / num_m) * BN;
+      int mb, nb;
+      tile_coords(t, num_m, num_n, p.band, mb, nb);
+      const int m0 = mb * (2 * BM) + rank * BM, n0 = nb * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
       // gated-residual epilogue: request of this lane's row, and whether the warp's rows share it
