@@ -34,7 +34,15 @@ DEFAULT_WORKLOAD = "cfg5_mixed8"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, transcribed from
 # the committed ncu summaries (profiles/); None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {}
+# Captured on cfg3_1024x2 (profiles/gemm_tcgen05_dram_traffic_cfg3_1024x2.md): 530 MB per launch averaged over the
+# four GEMMs of a block; traffic is proportional to T, so other workloads of the 3072-wide model scale by T / 9216.
+NCU_TRAFFIC_BYTES_PER_TOKEN_3072 = 530.0e6 / 9216
+
+
+def ncu_traffic(wl):
+    if wl.dims.hidden != 3072:
+        return None
+    return NCU_TRAFFIC_BYTES_PER_TOKEN_3072 * wl.total_tokens
 
 
 def measured_peaks():
@@ -258,7 +266,9 @@ def run_gpu(args):
                 "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": f"bf16 sustained, of {peaks['source']}",
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
                 "avg_launch_ms": gemm_ms / gemm_launches, "launches": gemm_launches,
-                "traffic": NCU_TRAFFIC_BYTES.get(wl.name)}
+                "traffic": ncu_traffic(wl),
+                "algorithmic_bytes": (T * H * 2 * 2 + 3 * H * H * 2 + T * 3 * H * 2 + H * H * 2 + T * H * 8 + T * H * 2 + H * F * 2
+                                      + T * F * 2 * 2 + F * H * 2 + T * H * 8) / 4.0}
 
     # ---------------------------------------------------------------- the oracle on the host cores
     run, n_img, desc = oracle_sample(wl)
