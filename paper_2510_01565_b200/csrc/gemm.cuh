@@ -170,10 +170,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (EPI == kEpiGateResidF32 && row_ok) my_req = find_request(seq, row);
       const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
       const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
+      // Residual rows of this tile do not depend on the accumulator: the first two 32-column chunks
+      // are requested before waiting for the MMAs, later chunks two iterations ahead.
+      const int cg = (lane & 7) * 4;
+      float4 xres[2][8];
+      auto load_resid = [&](int c, float4 (&x)[8]) {
+        const int col = n0 + c * 32 + cg;
+        if (EPI == kEpiGateResidF32 && col < p.N) {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int grow = m0 + quarter * 32 + it * 4 + (lane >> 3);
+            if (grow < p.M) x[it] = *reinterpret_cast<const float4*>(p.resid + static_cast<size_t>(grow) * p.N + col);
+          }
+        }
+      };
+      load_resid(0, xres[0]);
+      load_resid(1, xres[1]);
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-#pragma unroll 1
+#pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         __syncwarp();                          // tcgen05.ld is warp-collective: reconverge first
@@ -188,17 +204,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 32; ++i) st[lane * 33 + i] = __uint_as_float(r[i]);
           __syncwarp();
-          const int cg = (lane & 7) * 4, col = col0 + cg;   // N is a multiple of 64: the whole chunk is inside
+          const int col = col0 + cg;                        // N is a multiple of 64: the whole chunk is inside
           {
             const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(p.gate + req0 * p.gate_stride + col));
             float4 x[8];
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
-              const int grow = m0 + quarter * 32 + it * 4 + (lane >> 3);
-              if (grow < p.M) x[it] = *reinterpret_cast<const float4*>(p.resid + static_cast<size_t>(grow) * p.N + col);
-            }
+            for (int it = 0; it < 8; ++it) x[it] = xres[c & 1][it];
+            if (c + 2 < BN / 32) load_resid(c + 2, xres[c & 1]);
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
               const int rr = it * 4 + (lane >> 3);
