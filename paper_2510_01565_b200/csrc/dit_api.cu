@@ -179,7 +179,9 @@ cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float
   return cudaGetLastError();
 }
 
-size_t mod_smem_bytes(int C) { return (static_cast<size_t>(kModReqGroup) * C + 8 * kModReqGroup * kModCols) * sizeof(float); }
+size_t mod_smem_bytes(int C) {   // activations [G][C], later reused for the slice partials [slices][G][cols]
+  return std::max<size_t>(static_cast<size_t>(kModReqGroup) * C, static_cast<size_t>(kModSlices) * kModReqGroup * kModCols) * sizeof(float);
+}
 
 dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
                      float* out, cudaStream_t st) {

@@ -8,14 +8,17 @@ namespace dit {
 // ------------------------------------------------------------------------------------------------
 // adaLN modulation for all blocks at once:
 //   mod[r, b, j] = sum_c SiLU(cond[r, c]) * W_ada_b[c, j] + b_ada_b[j],   j in [0, 6H)
-// Bound by reading W_ada once (C x 6H bf16 per block).  A CTA owns 256 consecutive columns of one
-// block: 32 column groups (8 bf16 = 16 B per load) x 8 slices of the C range; slice partials are
+// Bound by reading W_ada once (C x 6H bf16 per block).  A CTA owns 128 consecutive columns of one
+// block: 16 column groups (8 bf16 = 16 B per load) x 16 slices of the C range; slice partials are
 // combined in shared memory in slice order, so the result does not depend on the number of requests.
+// The partials reuse the activation buffer, which keeps two CTAs resident per SM.
 // Requests are processed in groups of kModReqGroup to bound registers.
 // ------------------------------------------------------------------------------------------------
 constexpr int kModReqGroup = 8;
 constexpr int kModThreads = 256;
-constexpr int kModCols = 256;
+constexpr int kModCols = 128;
+constexpr int kModSlices = 16;
+constexpr int kModBatch = 12;
 
 struct ModParams {
   const __nv_bfloat16* cond;     // [R, C]
@@ -27,17 +30,17 @@ struct ModParams {
 };
 
 __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams p) {
-  extern __shared__ float sm[];                       // silu(cond) [G][C], then partials [8][G][256]
+  extern __shared__ float sm[];                       // silu(cond) [G][C]; afterwards reused for partials [16][G][128]
   const int cols_per_block = (p.N6 + kModCols - 1) / kModCols;
   const int blk = blockIdx.x / cols_per_block;
   const int col_base = (blockIdx.x % cols_per_block) * kModCols;
-  const int cg = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  const int cg = threadIdx.x & 15, slice = threadIdx.x >> 4;
   const int col = col_base + cg * 8;
   const __nv_bfloat16* w = p.w_ada0 + blk * p.w_block_stride;
   const float* bias = p.b_ada0 + blk * p.b_block_stride;
   float* s_act = sm;
-  float* s_part = sm + kModReqGroup * p.C;
-  const int c_per = (p.C + 7) / 8;
+  float* s_part = sm;
+  const int c_per = (p.C + kModSlices - 1) / kModSlices;
   const int c0 = slice * c_per, c1 = min(p.C, c0 + c_per);
 
   for (int r0 = 0; r0 < p.R; r0 += kModReqGroup) {
@@ -59,24 +62,42 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 #pragma unroll
       for (int k = 0; k < 8; ++k) acc[rr][k] = 0.f;
     if (col < p.N6) {
-#pragma unroll 4
-      for (int c = c0; c < c1; ++c) {
-        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(w + static_cast<size_t>(c) * p.N6 + col));
-        const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-        float wf[8];
+      // batches of kModBatch rows of W_ada: all loads of a batch are issued before any is used, so
+      // each thread keeps kModBatch x 16 bytes in flight (the kernel is bound by reading W_ada)
+      uint4 nxt[kModBatch];
+      auto fetch = [&](int cb) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          wf[2 * k] = __uint_as_float(u[k] << 16);
-          wf[2 * k + 1] = __uint_as_float(u[k] & 0xFFFF0000u);
-        }
+        for (int j = 0; j < kModBatch; ++j)
+          if (cb + j < c1) nxt[j] = __ldg(reinterpret_cast<const uint4*>(w + static_cast<size_t>(cb + j) * p.N6 + col));
+      };
+      fetch(c0);
+      for (int cb = c0; cb < c1; cb += kModBatch) {
+        uint4 raw[kModBatch];
 #pragma unroll
-        for (int rr = 0; rr < kModReqGroup; ++rr) {
-          const float a = s_act[rr * p.C + c];
+        for (int j = 0; j < kModBatch; ++j) raw[j] = nxt[j];
+        if (cb + kModBatch < c1) fetch(cb + kModBatch);          // next batch flies while this one is used
 #pragma unroll
-          for (int k = 0; k < 8; ++k) acc[rr][k] = fmaf(a, wf[k], acc[rr][k]);
+        for (int j = 0; j < kModBatch; ++j) {
+          if (cb + j < c1) {
+            const int c = cb + j;
+            const uint32_t u[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+            float wf[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              wf[2 * k] = __uint_as_float(u[k] << 16);
+              wf[2 * k + 1] = __uint_as_float(u[k] & 0xFFFF0000u);
+            }
+#pragma unroll
+            for (int rr = 0; rr < kModReqGroup; ++rr) {
+              const float a = s_act[rr * p.C + c];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) acc[rr][k] = fmaf(a, wf[k], acc[rr][k]);
+            }
+          }
         }
       }
     }
+    __syncthreads();                           // every thread is done with the activations: reuse the buffer
 #pragma unroll
     for (int rr = 0; rr < kModReqGroup; ++rr)
 #pragma unroll
@@ -87,7 +108,7 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
       if (col_base + cc < p.N6) {
         float v = 0.f;
 #pragma unroll
-        for (int sl = 0; sl < 8; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModCols + cc];
+        for (int sl = 0; sl < kModSlices; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModCols + cc];
         p.mod[(static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc] = v + bias[col_base + cc];
       }
     }
