@@ -45,6 +45,17 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
+// Non-blocking test of a phase (no suspension): the fast path of every wait.
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+
 // try_wait with a suspend-time hint (ns): the waiting thread is parked by the hardware instead of
 // re-polling, so it does not take issue slots from the warps that share its scheduler.
 __device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
@@ -72,6 +83,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   // try_wait suspends the thread in hardware until the phase completes or a short system limit
   // passes, so this loop is not a hot spin; the timer, the abort flag and the back-off only come
   // into play for waits far longer than any healthy one.
+  if (mbar_test_wait(bar, parity)) return true;          // already complete: no suspension round trip
   for (int i = 0; i < (1 << 16); ++i)
     if (mbar_try_wait_hint(bar, parity, DIT_MBAR_SUSPEND_NS)) return true;
   const uint64_t t0 = global_ns();
