@@ -216,6 +216,32 @@ def run_gpu(args):
     flops = wl.flops_per_step()
     tflops = flops / (ms_step * 1e-3) / 1e12
 
+    # ---------------------------------------------------------------- the same step replayed from a CUDA graph
+    # (the step neither allocates nor synchronises, so a caller can capture it; this removes the launch
+    # overhead that dominates the small-resolution steps)
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+        for _ in range(args.warmup):
+            g.replay()
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            g.replay()
+        e1.record(stream)
+        barrier()
+        graph_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    except Exception as exc:   # graph capture is a convenience figure, never the headline
+        sys.stderr.write(f"cuda graph timing skipped: {exc}\n")
+
     # ---------------------------------------------------------------- end to end with host buffers
     h_tok = torch.from_numpy(tok_bits.view(np.int16)).pin_memory()
     h_cond = torch.from_numpy(cond_bits.view(np.int16)).pin_memory()
@@ -292,6 +318,7 @@ def run_gpu(args):
             "roofline": roofline, "kernels": kern, "cpu_baseline": cpu,
             "e2e": {"value": img_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "cuda_graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms, "value": replicas.whole_job_rate(wl.image_tokens, world, graph_ms), "unit": UNIT},
             "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(line))
     if dist is not None:

@@ -289,3 +289,36 @@ def test_error_codes(B):
     assert float(out.min()) == 7.0
     ctx.dit_ctx_poll_status()
     ctx.close()
+
+
+def test_step_replays_from_a_cuda_graph(B):
+    """The step neither allocates nor synchronises, so a caller can capture it once and replay it:
+    this is what removes the launch overhead that dominates small-resolution steps (Section 3 of
+    the paper motivates batching small requests with exactly that overhead)."""
+    import torch
+    wl = W.make_custom("graph", W.SMALL, 2, [(256, 256, 0), (64, 64, 9)], seed=12, timestep_cond=False)
+    run = GpuRun(B, wl)
+    want = run.packed().clone()
+    out = torch.zeros_like(want)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run.ctx.dit_step_forward(run.tok, wl.token_lens, run.cond, 2, out=out)     # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run.ctx.dit_step_forward(run.tok, wl.token_lens, run.cond, 2, out=out)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, want)
+    # new token values in the same buffers: the replay follows them
+    run.tok.copy_(run.tok.flip(0).contiguous())
+    graph.replay()
+    torch.cuda.synchronize()
+    fresh = run.ctx.dit_step_forward(run.tok, wl.token_lens, run.cond, 2)
+    torch.cuda.synchronize()
+    assert torch.equal(out, fresh)
+    run.ctx.dit_ctx_poll_status()
+    run.close()
