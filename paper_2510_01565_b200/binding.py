@@ -42,6 +42,18 @@ class DitBlockWeights(C.Structure):
                                           "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
 
 
+SCHED_EXPORTS = ["dit_sched_allocate", "dit_sched_round"]
+
+
+class DitSchedOption(C.Structure):
+    _fields_ = [("steps", C.c_int32), ("gpus", C.c_int32), ("step_time", C.c_double)]
+
+
+class DitSchedRequest(C.Structure):
+    _fields_ = [("options", C.POINTER(DitSchedOption)), ("n_options", C.c_int32), ("t_min", C.c_double),
+                ("deadline", C.c_double)]
+
+
 class DitError(RuntimeError):
     def __init__(self, status: int, detail: str = ""):
         self.status = status
@@ -89,6 +101,12 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_read_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.dit_modulation_noalloc.restype = C.c_int
     lib.dit_modulation_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+    lib.dit_sched_allocate.restype = C.c_int
+    lib.dit_sched_allocate.argtypes = [C.POINTER(i32), C.POINTER(C.c_double), i32, i32, C.c_double,
+                                       C.POINTER(DitSchedOption), C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i32)]
+    lib.dit_sched_round.restype = C.c_int
+    lib.dit_sched_round.argtypes = [C.POINTER(DitSchedRequest), i32, i32, C.c_double, C.c_double, C.POINTER(i32),
+                                    C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     lib.dit_last_launch_count.restype = i64
     lib.dit_last_launch_count.argtypes = [vp]
     lib.dit_status_string.restype = C.c_char_p
@@ -97,6 +115,40 @@ def load_library() -> C.CDLL:
     lib.dit_last_error.argtypes = [vp]
     _lib = lib
     return lib
+
+
+def dit_sched_allocate(gpus: Sequence[int], step_time: Sequence[float], steps: int, time_budget: float):
+    """Returns (options [(steps, gpus, step_time)], gpu_time, feasible)."""
+    lib = load_library()
+    n = len(gpus)
+    g = (C.c_int32 * n)(*gpus)
+    t = (C.c_double * n)(*step_time)
+    out = (DitSchedOption * 2)()
+    n_out, feasible, cost = C.c_int32(), C.c_int32(), C.c_double()
+    st = lib.dit_sched_allocate(g, t, n, steps, time_budget, out, C.byref(n_out), C.byref(cost), C.byref(feasible))
+    if st != DIT_OK:
+        raise DitError(st)
+    return [(out[i].steps, out[i].gpus, out[i].step_time) for i in range(n_out.value)], cost.value, bool(feasible.value)
+
+
+def dit_sched_round(reqs, n_gpus: int, tau: float, t_now: float):
+    """reqs: list of (options [(steps, gpus, step_time)], t_min, deadline).
+    Returns (chosen option per request or -1, steps done per request, survivors, gpus used)."""
+    lib = load_library()
+    n = len(reqs)
+    keep = []
+    arr = (DitSchedRequest * max(n, 1))()
+    for i, (options, t_min, deadline) in enumerate(reqs):
+        o = (DitSchedOption * max(len(options), 1))(*[DitSchedOption(int(s), int(a), float(t)) for (s, a, t) in options])
+        keep.append(o)
+        arr[i] = DitSchedRequest(o, len(options), float(t_min), float(deadline))
+    chosen = (C.c_int32 * max(n, 1))()
+    done = (C.c_int32 * max(n, 1))()
+    surv, used = C.c_int32(), C.c_int32()
+    st = lib.dit_sched_round(arr, n, n_gpus, tau, t_now, chosen, done, C.byref(surv), C.byref(used))
+    if st != DIT_OK:
+        raise DitError(st)
+    return list(chosen[:n]), list(done[:n]), surv.value, used.value
 
 
 def dit_pack_requests(reqs: Sequence[Sequence]) -> Dict[str, np.ndarray]:

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdit.so")
-SOURCES = [os.path.join(CSRC, "dit_api.cu")]
+SOURCES = [os.path.join(CSRC, "dit_api.cu"), os.path.join(CSRC, "sched.cc")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 
