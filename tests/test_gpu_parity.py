@@ -322,3 +322,34 @@ def test_step_replays_from_a_cuda_graph(B):
     assert torch.equal(out, fresh)
     run.ctx.dit_ctx_poll_status()
     run.close()
+
+
+@pytest.mark.parametrize("dims,length", [(W.SMALL, 600), (W.LARGE, 400)])
+def test_growing_row_maximum_exercises_the_lazy_rescale(B, dims, length):
+    """Q = K = 2h makes every query's own key its by far largest score (about 2^29 times the rest
+    after exponentiation), so for rows beyond the first key tile the running maximum jumps in a
+    later tile and the accumulator in tensor memory has to be rescaled: the rarely taken path."""
+    n_text = length - 256
+    wl = W.make_custom("selfmatch", dims, 1, [(256, 256, n_text)], seed=13, timestep_cond=False)
+    H = dims.hidden
+    wq = np.zeros((H, 3 * H), dtype=np.float32)
+    idx = np.arange(H)
+    wq[idx, idx] = 2.0
+    wq[idx, H + idx] = 2.0
+    wq[idx, 2 * H + idx] = 1.0
+    wl.weights[0]["w_qkv"] = W.f32_to_bf16_bits(wq)
+    wl.weights[0]["b_qkv"] = W.f32_to_bf16_bits(np.zeros(3 * H, dtype=np.float32))
+    run = GpuRun(B, wl)
+    out = run.packed()
+    taps = {0: {}}
+    ref = oracle_requests(wl, [0], taps=taps)
+    # the scores really are this peaked: the self key carries almost all of the weight
+    qkv = taps[0]["qkv"]
+    d = dims.head_dim
+    s = (qkv[300, :d] @ qkv[:, H:H + d].T) / np.sqrt(d)
+    assert s.argmax() == 300 and s[300] - np.partition(s, -2)[-2] > 8 * np.log(2.0) * 1.5
+    got_a = run.ctx.dit_debug_tap("attn").cpu().numpy().astype(np.float64)
+    assert O.error_metric(got_a, taps[0]["a"]) <= TOL
+    check_request(run, out, 0, ref[0])
+    assert run.torch.equal(out, run.packed())
+    run.close()
