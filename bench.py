@@ -173,6 +173,12 @@ def run_gpu(args):
 
     wl = W.make_workload(args.workload, seed=args.seed)
     nb = wl.n_blocks
+    if args.depth:
+        # a deeper stack than the configuration draws (e.g. 57 blocks, the depth class of the models the
+        # paper serves): the drawn blocks' weights are loaded cyclically, which costs the same per block
+        nb = args.depth
+        wl.weights = [wl.weights[b % len(wl.weights)] for b in range(nb)]
+        wl.n_blocks = nb
     ctx = B.context_for(wl.dims, nb, wl.total_tokens, len(wl.requests))
     B.upload_weights(ctx, wl.weights)
     lens = wl.token_lens
@@ -309,7 +315,7 @@ def run_gpu(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
-            "config": {"workload": wl.name, "n_blocks": nb, "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
+            "config": {"workload": wl.name, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
                        "total_tokens": T, "image_tokens": wl.image_tokens, "hidden": H, "heads": wl.dims.n_heads,
                        "head_dim": wl.dims.head_dim, "mlp_hidden": F, "parallelism": f"replicas x{world}",
                        "l2": "weights and activations of a step exceed L2 (126 MB); no flush"},
@@ -332,6 +338,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--depth", type=int, default=0, help="run this many blocks instead of the configuration's (weights reused cyclically)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
