@@ -210,3 +210,66 @@ def make_workload(name: str, seed: int = 0, n_blocks: int | None = None,
                timestep_cond=(dims is LARGE), with_weights=with_weights)
     wl.n_blocks = nb
     return wl
+
+
+# --------------------------------------------------------------------------
+# inputs of a full denoising step (latent in, latent out) around the block stack
+# --------------------------------------------------------------------------
+LATENT_CHANNELS = 16     # latent z of an h x w request is [16, h/8, w/8] fp32
+VAE_FACTOR = 8
+PATCH_DIM = 64           # 16 channels x 2 x 2
+T_EMB_DIM = 256
+
+SHELL_WEIGHT_NAMES = ("w_in", "b_in", "w_t1", "b_t1", "w_t2", "b_t2", "w_fa", "b_fa", "w_out", "b_out")
+
+
+def draw_shell_weights(rng: np.random.Generator, dims: ModelDims) -> Dict[str, np.ndarray]:
+    """Embedding, timestep-MLP and final-layer tensors, row-major [in, out], bf16 bits.
+
+    The patch embedding is drawn at 1/sqrt(64) so that tokens come out at unit scale like the
+    N(0,1) token buffers of the step-only workloads; the rest at the 0.02 of the block weights.
+    """
+    h, c = dims.hidden, dims.cond_dim
+    shapes = {"w_in": (PATCH_DIM, h), "b_in": (h,), "w_t1": (T_EMB_DIM, c), "b_t1": (c,),
+              "w_t2": (c, c), "b_t2": (c,), "w_fa": (c, 2 * h), "b_fa": (2 * h,),
+              "w_out": (h, PATCH_DIM), "b_out": (PATCH_DIM,)}
+    return {k: _normal_bf16(rng, shapes[k], 0.125 if k == "w_in" else 0.02) for k in SHELL_WEIGHT_NAMES}
+
+
+@dataclass
+class StepInputs:
+    """Per-request inputs of full denoising steps, plus the model's tensors."""
+    dims: ModelDims
+    requests: List[Request]
+    latents: List[np.ndarray]          # per request [16, h/8, w/8] fp32, N(0,1)
+    texts: List[np.ndarray]            # per request [n_text, H] uint16 (bf16 bits), N(0,1)
+    pooled: np.ndarray                 # [R, C] fp32, N(0,1) (the prompt's pooled vector)
+    dsigmas: np.ndarray                # [R] fp32, sigma_next - sigma_cur of this step (negative)
+    shell: Dict[str, np.ndarray]
+    weights: List[Dict[str, np.ndarray]]
+
+    @property
+    def token_lens(self) -> List[int]:
+        return [r.n_tokens for r in self.requests]
+
+
+def make_step_inputs(dims: ModelDims, n_blocks: int, reqs: Sequence[Tuple[int, int, int]], seed: int = 0,
+                     n_steps: int = 50) -> StepInputs:
+    """Draw order: per request (step index, latent, text tokens, pooled), shell tensors, block tensors.
+
+    Each request sits at its own position of an n_steps-long schedule with sigma = 1 - i/n_steps
+    and t = 1000 sigma, as requests of a serving batch are at different steps of their schedules.
+    """
+    rng = np.random.default_rng(seed)
+    requests, latents, texts, pooled, dsig = [], [], [], [], []
+    for (hh, ww, n_text) in reqs:
+        i = int(rng.integers(0, n_steps))
+        sigma, sigma_next = 1.0 - i / n_steps, 1.0 - (i + 1) / n_steps
+        requests.append(Request(hh, ww, n_text, 1000.0 * sigma, i))
+        latents.append(rng.standard_normal(size=(LATENT_CHANNELS, hh // VAE_FACTOR, ww // VAE_FACTOR), dtype=np.float32))
+        texts.append(_normal_bf16(rng, (n_text, dims.hidden), 1.0))
+        pooled.append(rng.standard_normal(size=dims.cond_dim, dtype=np.float32))
+        dsig.append(np.float32(sigma_next - sigma))
+    shell = draw_shell_weights(rng, dims)
+    weights = [draw_block_weights(rng, dims) for _ in range(n_blocks)]
+    return StepInputs(dims, requests, latents, texts, np.stack(pooled), np.asarray(dsig, dtype=np.float32), shell, weights)

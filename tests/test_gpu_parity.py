@@ -41,7 +41,7 @@ def oracle_requests(wl, which, n_blocks=None, taps=None):
     return xs
 
 
-class GpuRun:
+class DeviceRun:
     def __init__(self, B, wl, n_blocks=None, max_requests=None):
         import torch
         self.torch, self.B, self.wl = torch, B, wl
@@ -88,7 +88,7 @@ def check_packed_equals_alone(run, out, requests=None):
 # ----------------------------------------------------------------------------- the five configurations
 def test_cfg1_small_block_full_parity_and_taps(B):
     wl = W.make_workload("cfg1_small_256")
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     taps = {0: {}}
     ref = oracle_requests(wl, [0], taps=taps)
@@ -108,7 +108,7 @@ def test_cfg1_small_block_full_parity_and_taps(B):
 
 def test_cfg2_512_four_blocks(B):
     wl = W.make_workload("cfg2_512")
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     check_request(run, out, 0, oracle_requests(wl, [0])[0])
     run.close()
@@ -116,7 +116,7 @@ def test_cfg2_512_four_blocks(B):
 
 def test_cfg3_1024_two_requests_packed(B):
     wl = W.make_workload("cfg3_1024x2")
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     check_packed_equals_alone(run, out)
     # full 4-block oracle on the second request (it sits at a non-zero packed offset)
@@ -126,7 +126,7 @@ def test_cfg3_1024_two_requests_packed(B):
 
 def test_cfg4_2048_long_sequence(B):
     wl = W.make_workload("cfg4_2048")
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     # one block at full length against oracle rows the CPU can produce one by one
     out1 = run.packed(n_blocks=1)
     L = wl.token_lens[0]
@@ -147,7 +147,7 @@ def test_cfg4_2048_long_sequence(B):
 def test_cfg5_mixed_resolution_eight_requests(B):
     wl = W.make_workload("cfg5_mixed8")
     assert [r.height for r in wl.requests] == [1024, 512, 256, 256, 1024, 2048, 1024, 1024]
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     assert bool(run.torch.isfinite(out).all())
     check_packed_equals_alone(run, out)
@@ -175,7 +175,7 @@ def test_cfg5_mixed_resolution_eight_requests(B):
 ])
 def test_ragged_lengths_one_block(B, dims, reqs):
     wl = W.make_custom("ragged", dims, 2, [(h, w, t) for (h, w, t) in reqs], seed=3)
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     ref = oracle_requests(wl, range(len(reqs)))
     for r in range(len(reqs)):
@@ -188,7 +188,7 @@ def test_sixty_four_requests(B):
     rng = np.random.default_rng(5)
     reqs = [(16, 16, int(rng.integers(0, 40))) for _ in range(64)]
     wl = W.make_custom("many", W.SMALL, 1, reqs, seed=4, timestep_cond=False)
-    run = GpuRun(B, wl, max_requests=64)
+    run = DeviceRun(B, wl, max_requests=64)
     out = run.packed()
     ref = oracle_requests(wl, range(64))
     for r in range(64):
@@ -204,7 +204,7 @@ def test_zero_gate_returns_input_exactly(B):
         for i in (2, 5):
             w["w_ada"][:, i * H:(i + 1) * H] = 0
             w["b_ada"][i * H:(i + 1) * H] = 0
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed().cpu().numpy()
     np.testing.assert_array_equal(out, W.bf16_bits_to_f32(wl.packed_tokens()))
     run.close()
@@ -212,7 +212,7 @@ def test_zero_gate_returns_input_exactly(B):
 
 def test_row_permutation_equivariance(B):
     wl = W.make_custom("perm", W.SMALL, 1, [(256, 256, 44)], seed=7, timestep_cond=False)
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed().cpu().numpy()
     perm = np.random.default_rng(0).permutation(wl.total_tokens)
     tokp = run.tok[run.torch.from_numpy(perm).cuda()].contiguous()
@@ -243,7 +243,7 @@ def test_null_biases_mean_zero(B):
 def test_pack_tokens_and_host_entry_point(B):
     import torch
     wl = W.make_custom("pack", W.SMALL, 1, [(64, 64, 7), (16, 16, 0), (96, 32, 100)], seed=9, timestep_cond=False)
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     per_req = [B.bits_to_cuda_bf16(t) for t in wl.tokens]
     packed = run.ctx.dit_pack_tokens(per_req)
     torch.cuda.synchronize()
@@ -297,7 +297,7 @@ def test_step_replays_from_a_cuda_graph(B):
     the paper motivates batching small requests with exactly that overhead)."""
     import torch
     wl = W.make_custom("graph", W.SMALL, 2, [(256, 256, 0), (64, 64, 9)], seed=12, timestep_cond=False)
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     want = run.packed().clone()
     out = torch.zeros_like(want)
     side = torch.cuda.Stream()
@@ -339,7 +339,7 @@ def test_growing_row_maximum_exercises_the_lazy_rescale(B, dims, length):
     wq[idx, 2 * H + idx] = 1.0
     wl.weights[0]["w_qkv"] = W.f32_to_bf16_bits(wq)
     wl.weights[0]["b_qkv"] = W.f32_to_bf16_bits(np.zeros(3 * H, dtype=np.float32))
-    run = GpuRun(B, wl)
+    run = DeviceRun(B, wl)
     out = run.packed()
     taps = {0: {}}
     ref = oracle_requests(wl, [0], taps=taps)
