@@ -77,7 +77,7 @@ typedef struct {
 typedef struct {
   int32_t height, width;  /* pixels, positive multiples of 16 */
   int32_t n_text_tokens;  /* >= 0; appended after the image tokens of the request */
-  float timestep;         /* t of this step; carried for the caller, the cond vector already encodes it */
+  float timestep;         /* t of this step; read by dit_timestep_cond / dit_denoise_step, else carried */
   int32_t step_index;     /* which of the request's S_i steps this is; carried for the caller */
 } dit_request;
 
@@ -93,7 +93,8 @@ typedef struct {
 
 /* Bytes of device workspace a context of this configuration needs (0 if the configuration is
  * invalid).  Covers converted weights for max_blocks blocks, the fp32 residual stream, the
- * intermediate activations, the modulation vectors and staging for dit_step_forward_host. */
+ * intermediate activations, the modulation vectors, staging for dit_step_forward_host and the
+ * tensors and intermediates of the shell calls (dit_load_shell_weights and below). */
 size_t dit_workspace_bytes(const dit_config *cfg);
 
 /* Creates a context on the current device.  `workspace` is device memory, 1024-byte aligned, at
@@ -181,7 +182,73 @@ dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *laun
 dit_status dit_modulation_noalloc(const void *cond, const void *w_ada, const void *b_ada, int32_t n_requests,
                                   int32_t cond_dim, int32_t hidden, float *mod_out, void *stream);
 
-/* Number of kernel launches issued by the last dit_step_forward on this context. */
+/* ------------------------------------------------------------------------------------------------
+ * The rest of a denoising step around the block stack.  In the paper a request's latent is the only
+ * state that lives from one step to the next and the only thing that moves between workers
+ * (Section 4, latent transfer between rounds); a step takes the latent, runs the transformer over
+ * all of its tokens (Section 2) and the sampler writes the next latent.  The paper leaves these
+ * parts to the model code it serves; the forms here are the usual ones of latent DiTs:
+ *
+ *   latent z_r   fp32 [16, h/8, w/8]; 2 x 2 patches, flattened in (channel, dy, dx) order to 64
+ *                numbers, patches in row-major (py, px) order: one token per 16 x 16 pixels
+ *   tokens       image row (py, px): patch W_in + b_in + pos(py, px), rounded to bf16, where the
+ *                first H/2 channels of pos encode py and the last H/2 encode px, each half being
+ *                [sin(p w_k) | cos(p w_k)], w_k = 10000^(-k/(H/4)), k < H/4;
+ *                text rows: taken as given (already H wide), after the image rows of the request
+ *   cond         e(t) = [cos(t f_k) | sin(t f_k)], f_k = 10000^(-k/128), k < 128;
+ *                c = SiLU(e W_t1 + b_t1) W_t2 + b_t2 (+ pooled), rounded to bf16
+ *   final layer  (shift, scale) = SiLU(c) W_fa + b_fa;  y = LN(x)(1 + scale) + shift;
+ *                v_tok = y W_out + b_out for image rows; un-patchified into v shaped like z
+ *   sampler      explicit Euler step of the rectified-flow ODE: z <- z + dsigma * v,
+ *                dsigma = sigma_next - sigma_cur
+ *
+ * Buffers that hold one array per request are concatenated in request order: `latents` and
+ * `velocity` are device fp32, request r starting at element 64 * (image tokens of requests before
+ * r); `text_tokens` is device bf16 [sum of n_text_tokens, H] (may be NULL when that sum is 0).
+ * Requests are HOST arrays; height, width, n_text_tokens and timestep are read.  These calls need
+ * hidden % 64 == 0 (as everywhere) and cond_dim % 8 == 0.  All are asynchronous on `stream`,
+ * allocate nothing, and detect argument errors on the host before any launch.
+ * ------------------------------------------------------------------------------------------------ */
+#define DIT_LATENT_CHANNELS 16
+#define DIT_PATCH_DIM 64  /* 16 channels x 2 x 2 */
+#define DIT_T_EMB_DIM 256
+
+/* Device pointers, bf16, row-major [in, out]; a NULL bias means zero.
+ *   w_in [64, H]   b_in [H]      w_t1 [256, C]  b_t1 [C]     w_t2 [C, C]  b_t2 [C]
+ *   w_fa [C, 2H]   b_fa [2H]  (shift | scale)   w_out [H, 64]  b_out [64] */
+typedef struct {
+  const void *w_in, *b_in, *w_t1, *b_t1, *w_t2, *b_t2, *w_fa, *b_fa, *w_out, *b_out;
+} dit_shell_weights;
+
+/* Copies the ten tensors into the context (W_out is re-laid out as fp16 for the tensor-core
+ * kernel, biases widened to fp32).  DIT_ERR_SHAPE if cond_dim is not a multiple of 8. */
+dit_status dit_load_shell_weights(dit_ctx *ctx, const dit_shell_weights *w, void *stream);
+
+/* cond_out [n, C] bf16 (device) from the requests' timesteps; pooled is device fp32 [n, C] or NULL. */
+dit_status dit_timestep_cond(dit_ctx *ctx, const dit_request *requests, int32_t n, const float *pooled,
+                             void *cond_out, void *stream);
+
+/* packed_tokens [T, H] bf16 (device), T = sum over requests of image + text tokens. */
+dit_status dit_embed_latents(dit_ctx *ctx, const float *latents, const void *text_tokens,
+                             const dit_request *requests, int32_t n, void *packed_tokens, void *stream);
+
+/* x [T, H] fp32 (device; the output of dit_step_forward), cond [n, C] bf16 (device) -> velocity. */
+dit_status dit_final_layer(dit_ctx *ctx, const float *x, const dit_request *requests, int32_t n,
+                           const void *cond, float *velocity, void *stream);
+
+/* latents += dsigma[r] * velocity, request by request; dsigma is a HOST array [n]. */
+dit_status dit_sampler_update(dit_ctx *ctx, float *latents, const float *velocity, const dit_request *requests,
+                              int32_t n, const float *dsigma, void *stream);
+
+/* The whole step in one call: conditioning, embedding, blocks 0..n_blocks-1, final layer and the
+ * update of `latents` in place.  `velocity` (device, same layout) also receives v when not NULL.
+ * Intermediates live in the context's workspace (the packed tokens share the staging buffer of
+ * dit_step_forward_host).  DIT_ERR_NOT_LOADED without shell or block weights. */
+dit_status dit_denoise_step(dit_ctx *ctx, float *latents, const void *text_tokens, const dit_request *requests,
+                            int32_t n, const float *dsigma, const float *pooled, int32_t n_blocks,
+                            float *velocity, void *stream);
+
+/* Number of kernel launches issued by the last dit_step_forward or dit_denoise_step on this context. */
 int64_t dit_last_launch_count(const dit_ctx *ctx);
 
 const char *dit_status_string(dit_status s);

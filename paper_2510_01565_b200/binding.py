@@ -23,7 +23,9 @@ TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_host",
-           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
+           "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
+           "dit_denoise_step", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
 
 class DitConfig(C.Structure):
@@ -40,6 +42,11 @@ class DitRequest(C.Structure):
 class DitBlockWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o",
                                           "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
+
+
+class DitShellWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_in", "b_in", "w_t1", "b_t1", "w_t2", "b_t2", "w_fa", "b_fa",
+                                          "w_out", "b_out")]
 
 
 SCHED_EXPORTS = ["dit_sched_allocate", "dit_sched_round"]
@@ -101,6 +108,20 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_read_timing.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.dit_modulation_noalloc.restype = C.c_int
     lib.dit_modulation_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+    fp = C.POINTER(C.c_float)
+    rq = C.POINTER(DitRequest)
+    lib.dit_load_shell_weights.restype = C.c_int
+    lib.dit_load_shell_weights.argtypes = [vp, C.POINTER(DitShellWeights), vp]
+    lib.dit_timestep_cond.restype = C.c_int
+    lib.dit_timestep_cond.argtypes = [vp, rq, i32, vp, vp, vp]
+    lib.dit_embed_latents.restype = C.c_int
+    lib.dit_embed_latents.argtypes = [vp, vp, vp, rq, i32, vp, vp]
+    lib.dit_final_layer.restype = C.c_int
+    lib.dit_final_layer.argtypes = [vp, vp, rq, i32, vp, vp, vp]
+    lib.dit_sampler_update.restype = C.c_int
+    lib.dit_sampler_update.argtypes = [vp, vp, vp, rq, i32, fp, vp]
+    lib.dit_denoise_step.restype = C.c_int
+    lib.dit_denoise_step.argtypes = [vp, vp, vp, rq, i32, fp, vp, i32, vp, vp]
     lib.dit_sched_allocate.restype = C.c_int
     lib.dit_sched_allocate.argtypes = [C.POINTER(i32), C.POINTER(C.c_double), i32, i32, C.c_double,
                                        C.POINTER(DitSchedOption), C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i32)]
@@ -149,6 +170,18 @@ def dit_sched_round(reqs, n_gpus: int, tau: float, t_now: float):
     if st != DIT_OK:
         raise DitError(st)
     return list(chosen[:n]), list(done[:n]), surv.value, used.value
+
+
+def request_array(reqs: Sequence) -> "C.Array":
+    """reqs: (height, width, n_text[, timestep, step_index]) tuples, or objects with those attributes."""
+    arr = (DitRequest * max(len(reqs), 1))()
+    for i, r in enumerate(reqs):
+        if hasattr(r, "height"):
+            arr[i] = DitRequest(int(r.height), int(r.width), int(r.n_text_tokens), float(r.timestep), int(r.step_index))
+        else:
+            arr[i] = DitRequest(int(r[0]), int(r[1]), int(r[2]), float(r[3]) if len(r) > 3 else 0.0,
+                                int(r[4]) if len(r) > 4 else 0)
+    return arr
 
 
 def dit_pack_requests(reqs: Sequence[Sequence]) -> Dict[str, np.ndarray]:
@@ -281,6 +314,97 @@ class DitContext:
                                                    C.c_void_p(host_out.data_ptr()), self._stream(stream)))
         return host_out
 
+    # ------------------------------------------------------------------ shell around the block stack
+    @staticmethod
+    def _ptr(t) -> C.c_void_p:
+        return C.c_void_p(t.data_ptr()) if t is not None else None
+
+    def _f32(self, t, n=None):
+        assert t.is_cuda and t.dtype == self.torch.float32 and t.is_contiguous()
+        assert n is None or t.numel() == n
+        return t
+
+    def dit_load_shell_weights(self, weights: Dict[str, "object"], stream=None):
+        """weights: name -> CUDA bf16 tensor, [in, out] row-major; biases may be None."""
+        w = DitShellWeights()
+        keep = []
+        for name, _ in DitShellWeights._fields_:
+            t = weights.get(name)
+            if t is not None:
+                assert t.is_cuda and t.dtype == self.torch.bfloat16 and t.is_contiguous(), name
+                keep.append(t)
+            setattr(w, name, t.data_ptr() if t is not None else None)
+        self._check(self.lib.dit_load_shell_weights(self.handle, C.byref(w), self._stream(stream)))
+
+    def dit_timestep_cond(self, reqs, pooled=None, cond_out=None, stream=None):
+        """-> cond [n, C] bf16 cuda.  pooled: [n, C] fp32 cuda or None."""
+        torch = self.torch
+        n = len(reqs)
+        if pooled is not None:
+            self._f32(pooled, n * self.cond_dim)
+        if cond_out is None:
+            cond_out = torch.empty((n, self.cond_dim), dtype=torch.bfloat16, device="cuda")
+        self._check(self.lib.dit_timestep_cond(self.handle, request_array(reqs), n, self._ptr(pooled),
+                                               self._ptr(cond_out), self._stream(stream)))
+        return cond_out
+
+    def dit_embed_latents(self, latents, text_tokens, reqs, packed_tokens=None, stream=None):
+        """latents: flat fp32 cuda (requests concatenated); text_tokens: [sum n_text, H] bf16 cuda or None."""
+        torch = self.torch
+        n = len(reqs)
+        arr = request_array(reqs)
+        n_img = sum((arr[i].height // 16) * (arr[i].width // 16) for i in range(n))
+        n_txt = sum(arr[i].n_text_tokens for i in range(n))
+        self._f32(latents, 64 * n_img)
+        if text_tokens is not None:
+            assert text_tokens.is_cuda and text_tokens.dtype == torch.bfloat16 and text_tokens.is_contiguous()
+            assert text_tokens.shape == (n_txt, self.hidden)
+        if packed_tokens is None:
+            packed_tokens = torch.empty((n_img + n_txt, self.hidden), dtype=torch.bfloat16, device="cuda")
+        self._check(self.lib.dit_embed_latents(self.handle, self._ptr(latents), self._ptr(text_tokens), arr, n,
+                                               self._ptr(packed_tokens), self._stream(stream)))
+        return packed_tokens
+
+    def dit_final_layer(self, x, reqs, cond, velocity=None, stream=None):
+        """x [T, H] fp32 cuda, cond [n, C] bf16 cuda -> velocity, flat fp32 cuda in latent layout."""
+        torch = self.torch
+        n = len(reqs)
+        arr = request_array(reqs)
+        n_img = sum((arr[i].height // 16) * (arr[i].width // 16) for i in range(n))
+        self._f32(x)
+        assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous() and cond.shape == (n, self.cond_dim)
+        if velocity is None:
+            velocity = torch.empty(64 * n_img, dtype=torch.float32, device="cuda")
+        self._f32(velocity, 64 * n_img)
+        self._check(self.lib.dit_final_layer(self.handle, self._ptr(x), arr, n, self._ptr(cond), self._ptr(velocity),
+                                             self._stream(stream)))
+        return velocity
+
+    def dit_sampler_update(self, latents, velocity, reqs, dsigma, stream=None):
+        n = len(reqs)
+        ds = np.ascontiguousarray(np.asarray(dsigma, dtype=np.float32))
+        assert ds.shape == (n,)
+        self._f32(latents)
+        self._f32(velocity, latents.numel())
+        self._check(self.lib.dit_sampler_update(self.handle, self._ptr(latents), self._ptr(velocity), request_array(reqs), n,
+                                                ds.ctypes.data_as(C.POINTER(C.c_float)), self._stream(stream)))
+        return latents
+
+    def dit_denoise_step(self, latents, text_tokens, reqs, dsigma, pooled, n_blocks: int, velocity=None, stream=None):
+        """One full step in place on `latents` (flat fp32 cuda).  Returns latents."""
+        n = len(reqs)
+        ds = np.ascontiguousarray(np.asarray(dsigma, dtype=np.float32))
+        assert ds.shape == (n,)
+        self._f32(latents)
+        if velocity is not None:
+            self._f32(velocity, latents.numel())
+        if pooled is not None:
+            self._f32(pooled, n * self.cond_dim)
+        self._check(self.lib.dit_denoise_step(self.handle, self._ptr(latents), self._ptr(text_tokens), request_array(reqs), n,
+                                              ds.ctypes.data_as(C.POINTER(C.c_float)), self._ptr(pooled), n_blocks,
+                                              self._ptr(velocity), self._stream(stream)))
+        return latents
+
     def dit_ctx_poll_status(self):
         self._check(self.lib.dit_ctx_poll_status(self.handle))
 
@@ -344,6 +468,14 @@ def upload_weights(ctx: DitContext, blocks) -> None:
         ctx.dit_load_block_weights(b, dev)
         torch.cuda.synchronize()
         del dev
+
+
+def upload_shell_weights(ctx: DitContext, shell) -> None:
+    """shell: dict name -> numpy uint16 (bf16 bits)."""
+    import torch
+    dev = {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in shell.items()}
+    ctx.dit_load_shell_weights(dev)
+    torch.cuda.synchronize()
 
 
 def bits_to_cuda_bf16(bits: np.ndarray):

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "gemm.cuh"
+#include "shell.cuh"
 
 using namespace dit;
 
@@ -31,8 +32,13 @@ struct BlockLayout {
 // Offsets (bytes) inside the workspace.
 struct Layout {
   BlockLayout blk;
-  size_t weights, stream, h, qkv, a, u, mod, status, stage_tokens, stage_cond, stage_out, bytes;
+  size_t weights, stream, h, qkv, a, u, mod, status, stage_tokens, stage_cond, stage_out;
+  // tensors and intermediates of the shell around the block stack
+  size_t sh_w_in, sh_b_in, sh_w_t1, sh_b_t1, sh_w_t2, sh_b_t2, sh_w_fa, sh_b_fa, sh_w_out, sh_b_out;
+  size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok;
+  size_t bytes;
 };
+constexpr int kWoutRows = 256;   // W_out^T is stored zero-padded to one full weight tile of the GEMM
 
 bool config_ok(const dit_config* c) {
   if (!c) return false;
@@ -75,6 +81,21 @@ Layout make_layout(const dit_config& c) {
   L.stage_tokens = take(T * H * 2);
   L.stage_cond = take(R * C * 2);
   L.stage_out = take(T * H * 4);
+  L.sh_w_in = take(DIT_PATCH_DIM * H * 2);
+  L.sh_b_in = take(H * 4);
+  L.sh_w_t1 = take(DIT_T_EMB_DIM * C * 2);
+  L.sh_b_t1 = take(C * 4);
+  L.sh_w_t2 = take(C * C * 2);
+  L.sh_b_t2 = take(C * 4);
+  L.sh_w_fa = take(C * 2 * H * 2);
+  L.sh_b_fa = take(2 * H * 4);
+  L.sh_w_out = take(kWoutRows * H * 2);
+  L.sh_b_out = take(DIT_PATCH_DIM * 4);
+  L.sh_temb = take(R * DIT_T_EMB_DIM * 4);
+  L.sh_pre1 = take(R * C * 4);
+  L.sh_cond = take(R * C * 2);
+  L.sh_modfin = take(R * 2 * H * 4);
+  L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
   L.bytes = o;
   return L;
 }
@@ -94,6 +115,8 @@ struct dit_ctx {
   int num_sms;
   int gemm_pairs;                          // CTA pairs of the GEMM kernel that fit on the device at once
   BlockState* blocks;
+  bool shell_loaded;
+  CUtensorMap tm_wout;                     // W_out^T, fp16 [kWoutRows, H]
   int64_t last_launches;
   int last_T, last_R, last_nb;
   char err[256];
@@ -240,7 +263,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     mp.mod = mod; mp.R = n; mp.C = c.cond_dim; mp.N6 = 6 * H; mp.NB = n_blocks;
     const int grid = n_blocks * ((6 * H + kModCols - 1) / kModCols);
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_MODULATION, [&] {
-      modulation_kernel<<<grid, kModThreads, mod_smem_bytes(c.cond_dim), st>>>(mp);
+      modulation_kernel<kModInCondSilu><<<grid, kModThreads, mod_smem_bytes(c.cond_dim), st>>>(mp);
       return cudaGetLastError();
     }));
   }
@@ -362,6 +385,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   ctx->num_sms = sms;
   ctx->blocks = new (std::nothrow) BlockState[cfg->max_blocks];
+  ctx->shell_loaded = false;
   ctx->last_launches = 0;
   ctx->last_T = ctx->last_R = ctx->last_nb = 0;
   ctx->timing = false;
@@ -376,9 +400,12 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF32>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
-  opt_in(reinterpret_cast<const void*>(&modulation_kernel), mod_smem_bytes(kMaxCondDim));  // same for every context
+  opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>), mod_smem_bytes(kMaxCondDim));  // same for every context
+  opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32Silu>), mod_smem_bytes(kMaxCondDim));
+  opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32>), mod_smem_bytes(kMaxCondDim));
   if (e == cudaSuccess) {
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(sms & ~1); lc.blockDim = dim3(gemm_cfg::THREADS); lc.dynamicSmemBytes = gemm_cfg::SMEM_BYTES;
@@ -590,6 +617,233 @@ const char* dit_last_error(const dit_ctx* ctx) { return ctx ? ctx->err : ""; }
 
 }  // extern "C"
 
+// =============================================================================================== shell around the block stack
+namespace {
+
+// Packed-batch and per-request geometry from a HOST request array (same rules as dit_pack_requests).
+dit_status build_shell(dit_ctx* ctx, const dit_request* reqs, int n, const float* dsigma, SeqInfo* seq, ShellInfo* info) {
+  if (n > ctx->cfg.max_requests) return fail(ctx, DIT_ERR_CAPACITY, "n exceeds max_requests");
+  int32_t lens[DIT_MAX_REQUESTS];
+  long long total = 0;
+  info->img_cu[0] = 0; info->txt_cu[0] = 0;
+  for (int r = 0; r < n; ++r) {
+    const dit_request& q = reqs[r];
+    if (q.height <= 0 || q.width <= 0 || q.height % 16 || q.width % 16 || q.n_text_tokens < 0)
+      return fail(ctx, DIT_ERR_SHAPE, "resolution must be a positive multiple of 16 and the text length non-negative");
+    const long long n_img = static_cast<long long>(q.height / 16) * (q.width / 16);
+    total += n_img + q.n_text_tokens;
+    if (total > ctx->cfg.max_total_tokens) return fail(ctx, DIT_ERR_CAPACITY, "packed batch exceeds max_total_tokens");
+    lens[r] = static_cast<int32_t>(n_img + q.n_text_tokens);
+    info->img_cu[r + 1] = info->img_cu[r] + static_cast<int>(n_img);
+    info->txt_cu[r + 1] = info->txt_cu[r] + q.n_text_tokens;
+    info->gw[r] = q.width / 16;
+    info->t[r] = q.timestep;
+    info->dsigma[r] = dsigma ? dsigma[r] : 0.f;
+  }
+  if (!build_seq(lens, n, seq)) return fail(ctx, DIT_ERR_INTERNAL, "empty request");
+  return DIT_OK;
+}
+
+// out[r, :] = act(in[r, :]) W + b (+ addend[r, :]): the modulation kernel with one "block".
+template <int kIn>
+cudaError_t launch_small_linear(const void* in, const void* w, const float* b, const float* addend, float* out32,
+                                __nv_bfloat16* out16, int R, int K, int N, cudaStream_t st) {
+  ModParams mp{};
+  if (kIn == kModInCondSilu) mp.cond = static_cast<const __nv_bfloat16*>(in); else mp.in32 = static_cast<const float*>(in);
+  mp.w_ada0 = static_cast<const __nv_bfloat16*>(w);
+  mp.b_ada0 = b;
+  mp.mod = out32; mp.out16 = out16; mp.addend = addend;
+  mp.R = R; mp.C = K; mp.N6 = N; mp.NB = 1;
+  modulation_kernel<kIn><<<(N + kModCols - 1) / kModCols, kModThreads, mod_smem_bytes(K), st>>>(mp);
+  return cudaGetLastError();
+}
+
+dit_status cond_impl(dit_ctx* ctx, const ShellInfo& info, int n, const float* pooled, void* cond_out, cudaStream_t st) {
+  const int Cd = ctx->cfg.cond_dim;
+  float* temb = ctx->at<float>(ctx->lay.sh_temb);
+  float* pre1 = ctx->at<float>(ctx->lay.sh_pre1);
+  timestep_embed_kernel<<<n, kTEmbDim, 0, st>>>(info, temb);
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
+  DIT_CUDA_TRY(ctx, launch_small_linear<kModInF32>(temb, ctx->ws + ctx->lay.sh_w_t1, ctx->at<float>(ctx->lay.sh_b_t1), nullptr,
+                                                   pre1, nullptr, n, kTEmbDim, Cd, st));
+  DIT_CUDA_TRY(ctx, launch_small_linear<kModInF32Silu>(pre1, ctx->ws + ctx->lay.sh_w_t2, ctx->at<float>(ctx->lay.sh_b_t2), pooled,
+                                                       nullptr, static_cast<__nv_bfloat16*>(cond_out), n, Cd, Cd, st));
+  return DIT_OK;
+}
+
+dit_status embed_impl(dit_ctx* ctx, const float* latents, const void* text, const SeqInfo& seq, const ShellInfo& info,
+                      void* tokens, cudaStream_t st) {
+  const int H = ctx->cfg.hidden;
+  dim3 grid((seq.total + kEmbRows - 1) / kEmbRows, (H + kEmbCols - 1) / kEmbCols);
+  embed_latents_kernel<<<grid, kEmbThreads, 0, st>>>(latents, static_cast<const __nv_bfloat16*>(text),
+                                                     ctx->at<__nv_bfloat16>(ctx->lay.sh_w_in), ctx->at<float>(ctx->lay.sh_b_in),
+                                                     static_cast<__nv_bfloat16*>(tokens), H, seq, info);
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
+  return DIT_OK;
+}
+
+// Final adaLN + output projection, then un-patchify into `velocity` and/or the Euler update of `latents`.
+dit_status final_impl(dit_ctx* ctx, const float* x, const SeqInfo& seq, const ShellInfo& info, int n, const void* cond,
+                      float* velocity, float* latents, cudaStream_t st) {
+  const dit_config& c = ctx->cfg;
+  const int T = seq.total, H = c.hidden;
+  float* modfin = ctx->at<float>(ctx->lay.sh_modfin);
+  __half* h = ctx->at<__half>(ctx->lay.h);
+  float* vtok = ctx->at<float>(ctx->lay.sh_vtok);
+  CUtensorMap tm_h;
+  if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM)) return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  DIT_CUDA_TRY(ctx, launch_small_linear<kModInCondSilu>(cond, ctx->ws + ctx->lay.sh_w_fa, ctx->at<float>(ctx->lay.sh_b_fa), nullptr,
+                                                        modfin, nullptr, n, c.cond_dim, 2 * H, st));
+  DIT_CUDA_TRY(ctx, launch_ln<false>(x, nullptr, h, modfin, modfin + H, 2ll * H, T, H, c.ln_eps, seq, st));
+  GemmParams g{};
+  g.status = ctx->at<int>(ctx->lay.status);
+  g.M = T; g.N = DIT_PATCH_DIM; g.K = H;
+  g.bias = ctx->at<float>(ctx->lay.sh_b_out);
+  g.out32 = vtok;
+  DIT_CUDA_TRY(ctx, launch_gemm<kEpiBiasF32>(ctx, tm_h, ctx->tm_wout, g, seq, st));
+  const long long work = static_cast<long long>(T) * (DIT_PATCH_DIM / 2);
+  const int grid = static_cast<int>(std::min<long long>((work + 255) / 256, static_cast<long long>(ctx->num_sms) * 16));
+  unpatchify_update_kernel<<<grid, 256, 0, st>>>(vtok, velocity, latents, seq, info);
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
+  return DIT_OK;
+}
+
+dit_status check_shell_args(dit_ctx* ctx, const dit_request* reqs, int n) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (n < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "n is negative");
+  if (n > 0 && !reqs) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL requests");
+  if (n > 0 && !ctx->shell_loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "dit_load_shell_weights has not been called");
+  return DIT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+dit_status dit_load_shell_weights(dit_ctx* ctx, const dit_shell_weights* w, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (!w) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weights");
+  if (!w->w_in || !w->w_t1 || !w->w_t2 || !w->w_fa || !w->w_out) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weight matrix");
+  const size_t H = ctx->cfg.hidden, Cd = ctx->cfg.cond_dim;
+  if (Cd % 8) return fail(ctx, DIT_ERR_SHAPE, "the shell needs cond_dim to be a multiple of 8");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = ctx->lay;
+  ctx->shell_loaded = false;
+  auto copy = [&](size_t off, const void* src, size_t bytes) {
+    return cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyDeviceToDevice, st);
+  };
+  auto bias = [&](const void* src, size_t off, int n) {
+    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), ctx->at<float>(off), n);
+    return cudaGetLastError();
+  };
+  DIT_CUDA_TRY(ctx, copy(L.sh_w_in, w->w_in, DIT_PATCH_DIM * H * 2));
+  DIT_CUDA_TRY(ctx, copy(L.sh_w_t1, w->w_t1, DIT_T_EMB_DIM * Cd * 2));
+  DIT_CUDA_TRY(ctx, copy(L.sh_w_t2, w->w_t2, Cd * Cd * 2));
+  DIT_CUDA_TRY(ctx, copy(L.sh_w_fa, w->w_fa, Cd * 2 * H * 2));
+  DIT_CUDA_TRY(ctx, bias(w->b_in, L.sh_b_in, static_cast<int>(H)));
+  DIT_CUDA_TRY(ctx, bias(w->b_t1, L.sh_b_t1, static_cast<int>(Cd)));
+  DIT_CUDA_TRY(ctx, bias(w->b_t2, L.sh_b_t2, static_cast<int>(Cd)));
+  DIT_CUDA_TRY(ctx, bias(w->b_fa, L.sh_b_fa, static_cast<int>(2 * H)));
+  DIT_CUDA_TRY(ctx, bias(w->b_out, L.sh_b_out, DIT_PATCH_DIM));
+  // W_out [H, 64] bf16 -> fp16 [64, H], padded with zero rows up to one weight tile
+  DIT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->ws + L.sh_w_out, 0, kWoutRows * H * 2, st));
+  {
+    dim3 grid((DIT_PATCH_DIM + 31) / 32, static_cast<unsigned>((H + 31) / 32));
+    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w->w_out), ctx->at<__half>(L.sh_w_out),
+                                                       static_cast<int>(H), DIT_PATCH_DIM);
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+  }
+  if (!make_map(ctx, &ctx->tm_wout, ctx->ws + L.sh_w_out, H, kWoutRows, gemm_cfg::BN / 2))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+  ctx->shell_loaded = true;
+  return DIT_OK;
+}
+
+dit_status dit_timestep_cond(dit_ctx* ctx, const dit_request* reqs, int32_t n, const float* pooled, void* cond_out, void* stream) {
+  dit_status s = check_shell_args(ctx, reqs, n);
+  if (s != DIT_OK || n == 0) return s;
+  if (!cond_out) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  SeqInfo seq{}; ShellInfo info{};
+  s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
+  if (s != DIT_OK) return s;
+  return cond_impl(ctx, info, n, pooled, cond_out, static_cast<cudaStream_t>(stream));
+}
+
+dit_status dit_embed_latents(dit_ctx* ctx, const float* latents, const void* text_tokens, const dit_request* reqs, int32_t n,
+                             void* packed_tokens, void* stream) {
+  dit_status s = check_shell_args(ctx, reqs, n);
+  if (s != DIT_OK || n == 0) return s;
+  if (!latents || !packed_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  SeqInfo seq{}; ShellInfo info{};
+  s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
+  if (s != DIT_OK) return s;
+  if (info.txt_cu[n] > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
+  return embed_impl(ctx, latents, text_tokens, seq, info, packed_tokens, static_cast<cudaStream_t>(stream));
+}
+
+dit_status dit_final_layer(dit_ctx* ctx, const float* x, const dit_request* reqs, int32_t n, const void* cond, float* velocity,
+                           void* stream) {
+  dit_status s = check_shell_args(ctx, reqs, n);
+  if (s != DIT_OK || n == 0) return s;
+  if (!x || !cond || !velocity) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  SeqInfo seq{}; ShellInfo info{};
+  s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
+  if (s != DIT_OK) return s;
+  return final_impl(ctx, x, seq, info, n, cond, velocity, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+dit_status dit_sampler_update(dit_ctx* ctx, float* latents, const float* velocity, const dit_request* reqs, int32_t n,
+                              const float* dsigma, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (n < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "n is negative");
+  if (n == 0) return DIT_OK;
+  if (!latents || !velocity || !reqs || !dsigma) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  SeqInfo seq{}; ShellInfo info{};
+  dit_status s = build_shell(ctx, reqs, n, dsigma, &seq, &info);
+  if (s != DIT_OK) return s;
+  const long long total = 64ll * info.img_cu[n];
+  const int grid = static_cast<int>(std::min<long long>((total + 255) / 256, static_cast<long long>(ctx->num_sms) * 16));
+  euler_update_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(latents, velocity, info, n);
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
+  return DIT_OK;
+}
+
+dit_status dit_denoise_step(dit_ctx* ctx, float* latents, const void* text_tokens, const dit_request* reqs, int32_t n,
+                            const float* dsigma, const float* pooled, int32_t n_blocks, float* velocity, void* stream) {
+  dit_status s = check_shell_args(ctx, reqs, n);
+  if (s != DIT_OK || n == 0) return s;
+  if (!latents || !dsigma) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  if (n_blocks < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "n_blocks must be at least 1");
+  if (n_blocks > ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "n_blocks exceeds max_blocks");
+  for (int b = 0; b < n_blocks; ++b)
+    if (!ctx->blocks[b].loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "a block in [0, n_blocks) has no weights");
+  SeqInfo seq{}; ShellInfo info{};
+  s = build_shell(ctx, reqs, n, dsigma, &seq, &info);
+  if (s != DIT_OK) return s;
+  if (info.txt_cu[n] > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* cond = ctx->ws + ctx->lay.sh_cond;
+  void* tokens = ctx->ws + ctx->lay.stage_tokens;
+  float* x = ctx->at<float>(ctx->lay.stream);
+  int32_t lens[DIT_MAX_REQUESTS];
+  for (int r = 0; r < n; ++r) lens[r] = seq.cu[r + 1] - seq.cu[r];
+  s = cond_impl(ctx, info, n, pooled, cond, st);
+  if (s != DIT_OK) return s;
+  s = embed_impl(ctx, latents, text_tokens, seq, info, tokens, st);
+  if (s != DIT_OK) return s;
+  s = step_impl(ctx, tokens, lens, n, cond, n_blocks, x, st);       // the last block writes the residual stream in place
+  if (s != DIT_OK) return s;
+  s = final_impl(ctx, x, seq, info, n, cond, velocity, latents, st);
+  if (s != DIT_OK) return s;
+  ctx->last_launches += 3 + 1 + 4;
+  return DIT_OK;
+}
+
+}  // extern "C"
+
 // =============================================================================================== no-allocation entry point
 // adaLN modulation vectors without a context, a workspace or any allocation.  The context path keeps
 // the fp32 copy of the modulation bias in the caller's workspace; here that scratch is a fixed
@@ -620,7 +874,7 @@ cudaError_t noalloc_scratch_for_current_device(float** out) {
     e = cudaGetSymbolAddress(&p, g_noalloc_bias_scratch);
     if (e != cudaSuccess) return e;
     if (!p) return cudaErrorInvalidSymbol;
-    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(&modulation_kernel),
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>),
                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(mod_smem_bytes(kNoAllocMaxCond)));
     if (e != cudaSuccess) return e;
@@ -653,7 +907,7 @@ extern "C" dit_status dit_modulation_noalloc(const void* cond, const void* w_ada
   mp.b_ada0 = scratch;
   mp.w_block_stride = 0; mp.b_block_stride = 0;
   mp.mod = mod_out; mp.R = n_requests; mp.C = cond_dim; mp.N6 = n6; mp.NB = 1;
-  modulation_kernel<<<(n6 + kModCols - 1) / kModCols, kModThreads, mod_smem_bytes(cond_dim), st>>>(mp);
+  modulation_kernel<kModInCondSilu><<<(n6 + kModCols - 1) / kModCols, kModThreads, mod_smem_bytes(cond_dim), st>>>(mp);
   if (cudaGetLastError() != cudaSuccess) return DIT_ERR_CUDA;
   return DIT_OK;
 }

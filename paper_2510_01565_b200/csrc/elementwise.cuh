@@ -27,8 +27,17 @@ struct ModParams {
   long long w_block_stride, b_block_stride;
   float* mod;                    // [R, NB, 6H]
   int R, C, N6, NB;
+  // Used by the small linear layers around the block stack (NB = 1), NULL otherwise:
+  const float* in32;             // fp32 input [R, C] instead of `cond` (kIn = 1, 2)
+  const float* addend;           // [R, N6] added to the result
+  __nv_bfloat16* out16;          // result written as bf16 [R, N6] instead of `mod`
 };
 
+// kIn selects the input of the layer: 0 = SiLU(bf16 cond) (the adaLN modulation), 1 = SiLU(fp32 in32),
+// 2 = fp32 in32 as it is.
+enum ModInput : int { kModInCondSilu = 0, kModInF32Silu = 1, kModInF32 = 2 };
+
+template <int kIn>
 __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams p) {
   extern __shared__ float sm[];                       // silu(cond) [G][C]; afterwards reused for partials [16][G][128]
   const int cols_per_block = (p.N6 + kModCols - 1) / kModCols;
@@ -50,8 +59,9 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
       const int rr = i / p.C, cc = i % p.C;
       float v = 0.f;
       if (rr < g) {
-        const float x = __bfloat162float(p.cond[static_cast<size_t>(r0 + rr) * p.C + cc]);
-        v = x / (1.0f + __expf(-x));
+        const size_t at = static_cast<size_t>(r0 + rr) * p.C + cc;
+        const float x = kIn == kModInCondSilu ? __bfloat162float(p.cond[at]) : p.in32[at];
+        v = kIn == kModInF32 ? x : x / (1.0f + __expf(-x));
       }
       s_act[i] = v;
     }
@@ -109,7 +119,11 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
         float v = 0.f;
 #pragma unroll
         for (int sl = 0; sl < kModSlices; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModCols + cc];
-        p.mod[(static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc] = v + bias[col_base + cc];
+        v += bias[col_base + cc];
+        const size_t at = (static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc;
+        if (kIn != kModInCondSilu && p.addend) v += p.addend[at];
+        if (kIn != kModInCondSilu && p.out16) p.out16[at] = __float2bfloat16_rn(v);
+        else p.mod[at] = v;
       }
     }
   }

@@ -17,13 +17,14 @@
 //   kEpiBiasF16      out16 = acc + bias                                   (QKV projection)
 //   kEpiBiasGeluF16  out16 = gelu_tanh(acc + bias)                        (MLP up-projection)
 //   kEpiGateResidF32 out32 = resid + gate[request(row)] * (acc + bias)    (attention / MLP output)
+//   kEpiBiasF32      out32 = acc + bias                                   (output projection of the final layer)
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace dit {
 
-enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32 = 2 };
+enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32 = 2, kEpiBiasF32 = 3 };
 
 struct GemmParams {
   int M, N, K;
@@ -197,7 +198,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tmem_ld_wait();
         const int col0 = n0 + c * 32;
         if (col0 >= p.N) continue;             // warp-uniform
-        if (EPI == kEpiGateResidF32) {
+        if (EPI == kEpiGateResidF32 || EPI == kEpiBiasF32) {
           // Transpose through shared memory so that each global access covers whole 128-byte row
           // segments: lane -> (row it*4 + lane/8, columns (lane%8)*4 .. +3).
           float* st = epi_stage + (warp - 2) * EPI_STAGE_FLOATS;
@@ -208,24 +209,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           {
             const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(p.gate + req0 * p.gate_stride + col));
+            if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(p.gate + req0 * p.gate_stride + col));
             float4 x[8];
+            if (EPI == kEpiGateResidF32) {
 #pragma unroll
-            for (int it = 0; it < 8; ++it) x[it] = xres[c & 1][it];
-            if (c + 2 < BN / 32) load_resid(c + 2, xres[c & 1]);
+              for (int it = 0; it < 8; ++it) x[it] = xres[c & 1][it];
+              if (c + 2 < BN / 32) load_resid(c + 2, xres[c & 1]);
+            }
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
               const int rr = it * 4 + (lane >> 3);
               const int grow = m0 + quarter * 32 + rr;
               const int rq = __shfl_sync(0xffffffffu, my_req, rr);
               if (grow < p.M) {
-                if (!one_req) g = __ldg(reinterpret_cast<const float4*>(p.gate + rq * p.gate_stride + col));
+                if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(p.gate + rq * p.gate_stride + col));
                 const float* a = st + rr * 33 + cg;
                 float4 o;
-                o.x = x[it].x + g.x * (a[0] + b.x);
-                o.y = x[it].y + g.y * (a[1] + b.y);
-                o.z = x[it].z + g.z * (a[2] + b.z);
-                o.w = x[it].w + g.w * (a[3] + b.w);
+                if (EPI == kEpiGateResidF32) {
+                  o.x = x[it].x + g.x * (a[0] + b.x);
+                  o.y = x[it].y + g.y * (a[1] + b.y);
+                  o.z = x[it].z + g.z * (a[2] + b.z);
+                  o.w = x[it].w + g.w * (a[3] + b.w);
+                } else {
+                  o = make_float4(a[0] + b.x, a[1] + b.y, a[2] + b.z, a[3] + b.w);
+                }
                 *reinterpret_cast<float4*>(p.out32 + static_cast<size_t>(grow) * p.N + col) = o;
               }
             }
