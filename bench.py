@@ -264,6 +264,39 @@ def run_gpu(args):
     h2d = h_tok.numel() * 2 + h_cond.numel() * 2
     d2h = h_out.numel() * 4
 
+    # ---------------------------------------------------------------- the full step: latent in, latent out
+    # (conditioning, patch embedding, the same block stack, final layer, Euler update; the shell's
+    # tensors are drawn from their own generator so that the step-only inputs above are unchanged)
+    shell_rng = np.random.default_rng(args.seed + 1000)
+    B.upload_shell_weights(ctx, W.draw_shell_weights(shell_rng, wl.dims))
+    n_lat = 64 * wl.image_tokens
+    latents = torch.randn(n_lat, device="cuda", generator=torch.Generator(device="cuda").manual_seed(args.seed))
+    n_txt = sum(r.n_text_tokens for r in wl.requests)
+    text = torch.randn((n_txt, wl.dims.hidden), device="cuda").to(torch.bfloat16) if n_txt else None
+    pooled = torch.randn((len(wl.requests), wl.dims.cond_dim), device="cuda")
+    dsig = np.full(len(wl.requests), -0.02, dtype=np.float32)
+
+    def timed_ms(fn, reps):
+        fn()
+        barrier()
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1)) / reps
+
+    full_steps = max(1, min(args.steps, 5))
+    full_ms = timed_ms(lambda: ctx.dit_denoise_step(latents, text, wl.requests, dsig, pooled, nb), full_steps)
+    full_launches = ctx.dit_last_launch_count()
+    cond_dev = ctx.dit_timestep_cond(wl.requests, pooled)
+    shell_ms = {"timestep_cond": timed_ms(lambda: ctx.dit_timestep_cond(wl.requests, pooled, cond_out=cond_dev), 5),
+                "embed_latents": timed_ms(lambda: ctx.dit_embed_latents(latents, text, wl.requests, packed_tokens=tok), 5)}
+    vel = torch.empty_like(latents)
+    shell_ms["final_layer"] = timed_ms(lambda: ctx.dit_final_layer(out, wl.requests, cond_dev, velocity=vel), 5)
+    shell_ms["sampler_update"] = timed_ms(lambda: ctx.dit_sampler_update(latents, vel, wl.requests, dsig), 5)
+    ctx.dit_ctx_poll_status()
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -325,6 +358,10 @@ def run_gpu(args):
             "e2e": {"value": img_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "cuda_graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms, "value": replicas.whole_job_rate(wl.image_tokens, world, graph_ms), "unit": UNIT},
+            "full_step": {"what": "latent in, latent out: conditioning + patch embedding + the block stack + final layer + Euler update",
+                          "ms_per_step": full_ms, "value": replicas.whole_job_rate(wl.image_tokens, world, full_ms), "unit": UNIT,
+                          "steps": full_steps, "launches_per_step": full_launches, "shell_ms": shell_ms,
+                          "shell_share": sum(shell_ms.values()) / full_ms},
             "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(line))
     if dist is not None:
