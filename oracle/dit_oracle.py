@@ -20,8 +20,15 @@ design notes of the repository):
   * LayerNorm over the H channels, biased variance, eps inside the root,
     no learned affine;  modulate = LN(x) * (1 + scale) + shift;
   * one weight set for image and text tokens; softmax scale 1/sqrt(d);
-    no mask inside a request, no other request visible; no positional term;
+    no mask inside a request, no other request visible; no positional term
+    unless asked for (below);
   * GELU in its tanh form.
+
+Optional parts, off by default, for the model variants the paper serves (its
+FLUX / SD3 class models): per-head RMS-norm of queries and keys with a learned
+[d] scale, and a 2-D rotary position term on queries and keys (first d/8
+channels of a head unrotated, then a patch-row group and a patch-column group
+of equal size, adjacent channel pairs, base 10000; text tokens at (0, 0)).
 
 Every function works on fp64 arrays.  Nothing is tiled, fused or reordered
 beyond taking query rows in slabs to bound memory (each softmax row is still
@@ -30,7 +37,9 @@ the full definition over all keys of the request).
 Parity pins (tests/test_oracle_pins.py): hand-derived 2-token cases, softmax
 rows summing to one, zero gate => identity, row-permutation equivariance,
 packed (explicit block-diagonal mask) == each request alone, closed forms for
-LayerNorm / SiLU / GELU / modulation, Table 1 token counts for the packer.
+LayerNorm / SiLU / GELU / modulation, Table 1 token counts for the packer;
+RMS-norm and rotary hand cases, norm preservation and the relative-position
+property of the rotary term.
 """
 from __future__ import annotations
 
@@ -129,20 +138,75 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
     return out
 
 
+def rms_norm_heads(z: np.ndarray, g: np.ndarray, n_heads: int, eps: float) -> np.ndarray:
+    """RMS-norm of every head of every row: z_head / sqrt(mean(z_head^2) + eps) * g, g [d]."""
+    L, H = z.shape
+    zh = z.reshape(L, n_heads, H // n_heads)
+    ms = (zh ** 2).mean(axis=-1, keepdims=True)
+    return (zh / np.sqrt(ms + eps) * g).reshape(L, H)
+
+
+def rope_groups(d: int) -> Tuple[int, int]:
+    """(d_t, d_axis): the first d/8 channels of a head are not rotated (an index axis that stays at
+    position 0); the rest splits evenly into a patch-row group and a patch-column group."""
+    d_t = d // 8
+    return d_t, (d - d_t) // 2
+
+
+def rope_2d(z: np.ndarray, positions: np.ndarray, n_heads: int) -> np.ndarray:
+    """Rotary position term on every head.  positions [L, 2] = (patch row, patch column); text
+    tokens carry (0, 0).  In a group of n channels pair i = channels (2i, 2i+1) of the group turns by
+    the angle p * 10000^(-2i/n), p being the row for the first group and the column for the second."""
+    L, H = z.shape
+    d = H // n_heads
+    d_t, n = rope_groups(d)
+    out = z.reshape(L, n_heads, d).copy()
+    theta = 10000.0 ** (-2.0 * np.arange(n // 2, dtype=np.float64) / n)
+    for axis in range(2):
+        ang = positions[:, axis].astype(np.float64)[:, None] * theta[None, :]        # [L, n/2]
+        c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+        lo = d_t + axis * n
+        a, b = out[:, :, lo:lo + n:2].copy(), out[:, :, lo + 1:lo + n:2].copy()
+        out[:, :, lo:lo + n:2] = a * c - b * s
+        out[:, :, lo + 1:lo + n:2] = a * s + b * c
+    return out.reshape(L, H)
+
+
+def patch_positions(height: int, width: int, n_text: int) -> np.ndarray:
+    """[L, 2] (patch row, patch column) of a request's tokens: image tokens row-major, text at (0, 0)."""
+    gh, gw = height // PATCH_PIXELS, width // PATCH_PIXELS
+    py, px = np.meshgrid(np.arange(gh), np.arange(gw), indexing="ij")
+    img = np.stack([py.reshape(-1), px.reshape(-1)], axis=1)
+    return np.concatenate([img, np.zeros((n_text, 2), dtype=img.dtype)], axis=0)
+
+
 def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps: float,
-                  rows: np.ndarray | None = None, taps: dict | None = None) -> np.ndarray:
+                  rows: np.ndarray | None = None, taps: dict | None = None,
+                  positions: np.ndarray | None = None) -> np.ndarray:
     """One adaLN-Zero DiT block on one request.  x [L, H], cond [C] -> [L, H].
 
     With `rows`, only those output rows are produced (keys and values still
     come from every row of the request); used to sample outputs of long
     sequences.  `taps`, if given, receives the intermediates h1, qkv, a, x_mid,
     h2, u for per-kernel comparisons.
+
+    Two optional parts of the model variants: if `w` holds "q_norm" / "k_norm"
+    ([d] each), queries and keys are RMS-normed per head (same eps) before
+    attention; if `positions` [L, 2] is given, queries and keys then get the
+    2-D rotary term.  The taps' qkv is taken after both.
     """
     H = x.shape[1]
     shift_a, scale_a, gate_a, shift_m, scale_m, gate_m = adaln_modulation(cond, w["w_ada"], w["b_ada"])
     h = modulate(layer_norm(x, eps), shift_a, scale_a)
     qkv = h @ w["w_qkv"] + w["b_qkv"]
     q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+    if "q_norm" in w:
+        q = rms_norm_heads(q, w["q_norm"], n_heads, eps)
+        k = rms_norm_heads(k, w["k_norm"], n_heads, eps)
+    if positions is not None:
+        q, k = rope_2d(q, positions, n_heads), rope_2d(k, positions, n_heads)
+    if "q_norm" in w or positions is not None:
+        qkv = np.concatenate([q, k, v], axis=1)
     a = attention(q, k, v, n_heads, rows)
     xr = x if rows is None else x[rows]
     x_mid = xr + gate_a * (a @ w["w_o"] + w["b_o"])
@@ -155,20 +219,22 @@ def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps
 
 
 def stack_forward_alone(x: np.ndarray, cond: np.ndarray, blocks: Sequence[Weights],
-                        n_heads: int, eps: float) -> np.ndarray:
+                        n_heads: int, eps: float, positions: np.ndarray | None = None) -> np.ndarray:
     """A stack of blocks on one request run by itself."""
     for w in blocks:
-        x = block_forward(x, cond, w, n_heads, eps)
+        x = block_forward(x, cond, w, n_heads, eps, positions=positions)
     return x
 
 
 def step_forward(packed: np.ndarray, token_lens: Sequence[int], cond: np.ndarray,
-                 blocks: Sequence[Weights], n_heads: int, eps: float) -> np.ndarray:
+                 blocks: Sequence[Weights], n_heads: int, eps: float,
+                 positions: Sequence[np.ndarray] | None = None) -> np.ndarray:
     """One denoising step over a packed batch: each request through the stack on its own."""
     out = np.empty_like(packed)
     p = 0
     for r, l in enumerate(token_lens):
-        out[p:p + l] = stack_forward_alone(packed[p:p + l], cond[r], blocks, n_heads, eps)
+        out[p:p + l] = stack_forward_alone(packed[p:p + l], cond[r], blocks, n_heads, eps,
+                                           None if positions is None else positions[r])
         p += l
     return out
 

@@ -1,0 +1,131 @@
+"""Pins for the optional model-variant parts of the block oracle: per-head RMS-norm of queries and
+keys, and the 2-D rotary position term."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import dit_oracle as O
+
+
+def test_rms_norm_hand_cases():
+    # one head of 4: [3, 4, 0, 0] has mean square 25/4, so the normed vector is [1.2, 1.6, 0, 0]
+    z = np.array([[3.0, 4.0, 0.0, 0.0]])
+    assert np.allclose(O.rms_norm_heads(z, np.ones(4), 1, 0.0), [[1.2, 1.6, 0.0, 0.0]], atol=1e-15)
+    # the learned scale multiplies channel by channel
+    assert np.allclose(O.rms_norm_heads(z, np.array([2.0, -1.0, 5.0, 7.0]), 1, 0.0), [[2.4, -1.6, 0.0, 0.0]], atol=1e-15)
+    # two heads are normed separately: a constant head c becomes sign(c)
+    z = np.array([[5.0, 5.0, -0.01, -0.01]])
+    assert np.allclose(O.rms_norm_heads(z, np.ones(2), 2, 0.0), [[1.0, 1.0, -1.0, -1.0]], atol=1e-15)
+    # eps sits inside the root: a zero head stays zero, a head of 1s becomes 1/sqrt(1 + eps)
+    z = np.array([[0.0, 0.0, 1.0, 1.0]])
+    got = O.rms_norm_heads(z, np.ones(2), 2, 0.21)
+    assert np.allclose(got, [[0.0, 0.0, 1 / 1.1, 1 / 1.1]], atol=1e-15)
+    # scale invariance and unit mean square (eps = 0)
+    rng = np.random.default_rng(0)
+    z = rng.standard_normal((7, 96))
+    a = O.rms_norm_heads(z, np.ones(32), 3, 0.0)
+    assert np.allclose(a, O.rms_norm_heads(17.0 * z, np.ones(32), 3, 0.0), atol=1e-14)
+    assert np.allclose((a.reshape(7, 3, 32) ** 2).mean(-1), 1.0, atol=1e-14)
+
+
+def test_rope_groups_for_the_two_head_sizes():
+    assert O.rope_groups(128) == (16, 56)
+    assert O.rope_groups(64) == (8, 28)
+    assert O.rope_groups(32) == (4, 14)
+
+
+def test_rope_hand_case():
+    # one head of 32: channels 0..3 fixed, 4..17 turn with the row, 18..31 with the column.
+    z = np.zeros((1, 32))
+    z[0, 2] = 9.0             # unrotated group
+    z[0, 4], z[0, 5] = 1.0, 0.0       # row group, pair 0: frequency 1
+    z[0, 16], z[0, 17] = 0.0, 2.0     # row group, pair 6: frequency 10000^(-12/14)
+    z[0, 18], z[0, 19] = 3.0, 4.0     # column group, pair 0: frequency 1
+    py, px = 2, 5
+    out = O.rope_2d(z, np.array([[py, px]]), 1)[0]
+    assert out[2] == 9.0
+    assert out[4] == pytest.approx(math.cos(2.0), abs=1e-15) and out[5] == pytest.approx(math.sin(2.0), abs=1e-15)
+    a = py * 10000.0 ** (-12.0 / 14.0)
+    assert out[16] == pytest.approx(-2.0 * math.sin(a), abs=1e-15) and out[17] == pytest.approx(2.0 * math.cos(a), abs=1e-15)
+    assert out[18] == pytest.approx(3 * math.cos(5.0) - 4 * math.sin(5.0), abs=1e-14)
+    assert out[19] == pytest.approx(3 * math.sin(5.0) + 4 * math.cos(5.0), abs=1e-14)
+    untouched = [i for i in range(32) if i not in (2, 4, 5, 16, 17, 18, 19)]
+    assert np.array_equal(out[untouched], np.zeros(len(untouched)))
+
+
+def test_rope_is_a_rotation_and_encodes_relative_position():
+    rng = np.random.default_rng(1)
+    heads, d = 3, 64
+    q, k = rng.standard_normal((1, heads * d)), rng.standard_normal((1, heads * d))
+    # position (0, 0) (text tokens) leaves the vector as it is
+    assert np.array_equal(O.rope_2d(q, np.array([[0, 0]]), heads), q)
+    # per-head norms survive any position
+    r = O.rope_2d(q, np.array([[37, 120]]), heads)
+    assert np.allclose((r.reshape(heads, d) ** 2).sum(-1), (q.reshape(heads, d) ** 2).sum(-1), rtol=1e-13)
+    # the score of a query at p and a key at p' depends on p - p' only, head by head
+    def scores(pq, pk):
+        a = O.rope_2d(q, np.array([pq]), heads).reshape(heads, d)
+        b = O.rope_2d(k, np.array([pk]), heads).reshape(heads, d)
+        return (a * b).sum(-1)
+    base = scores((10, 3), (4, 9))
+    assert np.allclose(scores((10 + 50, 3 + 20), (4 + 50, 9 + 20)), base, atol=1e-12)
+    assert not np.allclose(scores((10, 3), (5, 9)), base, atol=1e-3)
+    # rows and columns act on different channels: moving only the column leaves the row group's part alone
+    a = O.rope_2d(q, np.array([[6, 1]]), heads).reshape(heads, d)
+    b = O.rope_2d(q, np.array([[6, 77]]), heads).reshape(heads, d)
+    assert np.array_equal(a[:, :8 + 28], b[:, :8 + 28]) and not np.allclose(a[:, 8 + 28:], b[:, 8 + 28:])
+
+
+def test_patch_positions():
+    p = O.patch_positions(32, 48, 2)            # 2 x 3 patches, then two text tokens
+    assert p.tolist() == [[0, 0], [0, 1], [0, 2], [1, 0], [1, 1], [1, 2], [0, 0], [0, 0]]
+
+
+def _block(rng, H, F, C, d=None):
+    w = {"w_ada": rng.standard_normal((C, 6 * H)) * 0.1, "b_ada": rng.standard_normal(6 * H) * 0.1,
+         "w_qkv": rng.standard_normal((H, 3 * H)) * 0.2, "b_qkv": rng.standard_normal(3 * H) * 0.1,
+         "w_o": rng.standard_normal((H, H)) * 0.2, "b_o": np.zeros(H),
+         "w_fc1": rng.standard_normal((H, F)) * 0.2, "b_fc1": np.zeros(F),
+         "w_fc2": rng.standard_normal((F, H)) * 0.2, "b_fc2": np.zeros(H)}
+    if d:
+        w["q_norm"] = 1.0 + 0.1 * rng.standard_normal(d)
+        w["k_norm"] = 1.0 + 0.1 * rng.standard_normal(d)
+    return w
+
+
+def test_block_with_variants_reduces_to_the_plain_block():
+    rng = np.random.default_rng(2)
+    H, heads, L = 64, 2, 6
+    w = _block(rng, H, 128, 8)
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(8)
+    plain = O.block_forward(x, cond, w, heads, 1e-6)
+    # all tokens at position (0, 0): the rotary term is the identity
+    assert np.array_equal(O.block_forward(x, cond, w, heads, 1e-6, positions=np.zeros((L, 2), dtype=int)), plain)
+    # a common shift of all positions changes no score, hence nothing
+    pos = np.array([[0, 0], [0, 1], [1, 0], [1, 1], [2, 0], [2, 1]])
+    a = O.block_forward(x, cond, w, heads, 1e-6, positions=pos)
+    b = O.block_forward(x, cond, w, heads, 1e-6, positions=pos + np.array([7, 30]))
+    assert np.allclose(a, b, atol=1e-11) and not np.allclose(a, plain, atol=1e-3)
+    # RMS-norm of q and k makes the block blind to the scale of W_q and W_k (eps = 0, zero q/k bias)
+    wn = dict(_block(rng, H, 128, 8, d=32))
+    wn["b_qkv"] = np.concatenate([np.zeros(2 * H), wn["b_qkv"][2 * H:]])
+    ref = O.block_forward(x, cond, wn, heads, 0.0, positions=pos)
+    ws = dict(wn)
+    ws["w_qkv"] = np.concatenate([3.0 * wn["w_qkv"][:, :H], 0.25 * wn["w_qkv"][:, H:2 * H], wn["w_qkv"][:, 2 * H:]], axis=1)
+    # eps = 0 also in LayerNorm here; harmless for random rows
+    assert np.allclose(O.block_forward(x, cond, ws, heads, 0.0, positions=pos), ref, atol=1e-11)
+
+
+def test_taps_hold_normed_and_rotated_queries():
+    rng = np.random.default_rng(3)
+    H, heads, L = 64, 2, 4
+    w = _block(rng, H, 128, 8, d=32)
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(8)
+    pos = np.array([[0, 0], [0, 1], [1, 0], [1, 1]])
+    taps = {}
+    O.block_forward(x, cond, w, heads, 1e-6, taps=taps, positions=pos)
+    raw = taps["h1"] @ w["w_qkv"] + w["b_qkv"]
+    want_q = O.rope_2d(O.rms_norm_heads(raw[:, :H], w["q_norm"], heads, 1e-6), pos, heads)
+    assert np.array_equal(taps["qkv"][:, :H], want_q)
+    assert np.array_equal(taps["qkv"][:, 2 * H:], raw[:, 2 * H:])      # values are neither normed nor rotated
