@@ -68,8 +68,20 @@ typedef struct {
   int32_t max_total_tokens; /* capacity T_max of one packed batch */
   int32_t max_requests;     /* capacity R_max, <= DIT_MAX_REQUESTS */
   float ln_eps;             /* LayerNorm epsilon (1e-6 in every benchmark configuration) */
-  uint32_t flags;           /* reserved, must be 0 */
+  uint32_t flags;           /* DIT_FLAG_* bits; 0 = the plain block */
 } dit_config;
+
+/* Model-variant parts of the block, as in the FLUX / SD3 class models the paper serves (Section 6.1
+ * lists them; the paper does not restate their layers).  Both act on queries and keys only, after the
+ * QKV projection and before attention, and are fused into that projection's epilogue.
+ *   DIT_FLAG_QK_RMSNORM  per head: q <- q / sqrt(mean(q^2) + ln_eps) * q_norm, same for k with k_norm
+ *   DIT_FLAG_ROPE_2D     2-D rotary term per head: the first d/8 channels stay; the next (d - d/8)/2
+ *                        turn with the token's patch row, the last (d - d/8)/2 with its patch column;
+ *                        in a group of n channels, pair (2i, 2i+1) turns by p * 10000^(-2i/n).  Text
+ *                        tokens sit at (0, 0).  Needs the requests' geometry: dit_step_forward_requests
+ *                        or dit_denoise_step (dit_step_forward returns DIT_ERR_INVALID_ARG). */
+#define DIT_FLAG_QK_RMSNORM 1u
+#define DIT_FLAG_ROPE_2D 2u
 
 /* One request of the paper's problem statement (Section 3): an image resolution, a position in
  * its denoising schedule and the diffusion time of this step.  Image tokens = (height/16) *
@@ -86,9 +98,11 @@ typedef struct {
  *   w_qkv [H, 3H]  b_qkv [3H]   columns: Q | K | V
  *   w_o   [H, H]   b_o   [H]
  *   w_fc1 [H, F]   b_fc1 [F]
- *   w_fc2 [F, H]   b_fc2 [H] */
+ *   w_fc2 [F, H]   b_fc2 [H]
+ *   q_norm [d]     k_norm [d]   RMS-norm scales (read with DIT_FLAG_QK_RMSNORM; NULL means ones) */
 typedef struct {
   const void *w_ada, *b_ada, *w_qkv, *b_qkv, *w_o, *b_o, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+  const void *q_norm, *k_norm;
 } dit_block_weights;
 
 /* Bytes of device workspace a context of this configuration needs (0 if the configuration is
@@ -132,6 +146,13 @@ dit_status dit_pack_tokens(dit_ctx *ctx, const void *const *per_request_tokens, 
 dit_status dit_step_forward(dit_ctx *ctx, const void *packed_tokens, const int32_t *per_request_token_lens,
                             int32_t n_requests, const void *per_request_cond, int32_t n_blocks, float *out,
                             void *stream);
+
+/* The same step with the batch described by requests (HOST array; height, width and n_text_tokens
+ * are read, token lengths follow from them as in dit_pack_requests).  The only entry point of the
+ * block stack that can run with DIT_FLAG_ROPE_2D, since it knows every token's patch row and column. */
+dit_status dit_step_forward_requests(dit_ctx *ctx, const void *packed_tokens, const dit_request *requests,
+                                     int32_t n_requests, const void *per_request_cond, int32_t n_blocks,
+                                     float *out, void *stream);
 
 /* Same step with HOST buffers: copies tokens and cond to the device, runs the step, copies `out`
  * back, all on `stream`, and returns after the stream has drained (out is valid on return).

@@ -133,12 +133,14 @@ def euler_update(z: np.ndarray, v: np.ndarray, dsigma: float) -> np.ndarray:
 
 def denoise_step(latents: Sequence[np.ndarray], texts: Sequence[np.ndarray], timesteps: Sequence[float],
                  dsigmas: Sequence[float], pooled: Sequence[np.ndarray | None], shell: ShellWeights,
-                 block_ws: Sequence[blocks.Weights], n_heads: int, eps: float):
+                 block_ws: Sequence[blocks.Weights], n_heads: int, eps: float, rope: bool = False):
     """One full step of every request (each on its own).  Returns (new latents, velocities, taps).
 
     texts[r] is [n_text_r, H] (already bf16-representable) or an empty array.
     taps holds the intermediate results the parity tests compare: cond (bf16-rounded), tokens
-    (bf16-rounded, image then text rows) and the stack output, per request.
+    (bf16-rounded, image then text rows) and the stack output, per request.  With `rope` the blocks
+    apply the 2-D rotary term at the tokens' patch positions (RMS-norm of queries and keys is
+    switched on by the block weights holding q_norm / k_norm).
     """
     new_latents, velocities, taps = [], [], []
     for z, txt, t, ds, pl in zip(latents, texts, timesteps, dsigmas, pooled):
@@ -146,7 +148,8 @@ def denoise_step(latents: Sequence[np.ndarray], texts: Sequence[np.ndarray], tim
         cond = round_to_bf16(timestep_cond(t, pl, shell))
         img = round_to_bf16(embed_latent(z, shell, hidden))
         tokens = img if txt.shape[0] == 0 else np.concatenate([img, txt], axis=0)
-        x = blocks.stack_forward_alone(tokens, cond, block_ws, n_heads, eps)
+        pos = blocks.patch_positions(z.shape[1] * VAE_FACTOR, z.shape[2] * VAE_FACTOR, txt.shape[0]) if rope else None
+        x = blocks.stack_forward_alone(tokens, cond, block_ws, n_heads, eps, positions=pos)
         v_tok = final_layer(x[:img.shape[0]], cond, shell, eps)
         v = unpatchify(v_tok, z.shape[1], z.shape[2])
         new_latents.append(euler_update(z, v, ds))

@@ -16,13 +16,15 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdit.so")
 
 DIT_OK = 0
+DIT_FLAG_QK_RMSNORM = 1
+DIT_FLAG_ROPE_2D = 2
 STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
                 "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
 KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
-           "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_host",
+           "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
            "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
            "dit_denoise_step", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
@@ -41,7 +43,7 @@ class DitRequest(C.Structure):
 
 class DitBlockWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o",
-                                          "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
+                                          "w_fc1", "b_fc1", "w_fc2", "b_fc2", "q_norm", "k_norm")]
 
 
 class DitShellWeights(C.Structure):
@@ -110,6 +112,8 @@ def load_library() -> C.CDLL:
     lib.dit_modulation_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     fp = C.POINTER(C.c_float)
     rq = C.POINTER(DitRequest)
+    lib.dit_step_forward_requests.restype = C.c_int
+    lib.dit_step_forward_requests.argtypes = [vp, vp, rq, i32, vp, i32, vp, vp]
     lib.dit_load_shell_weights.restype = C.c_int
     lib.dit_load_shell_weights.argtypes = [vp, C.POINTER(DitShellWeights), vp]
     lib.dit_timestep_cond.restype = C.c_int
@@ -212,14 +216,15 @@ class DitContext:
     """Owns a workspace tensor and a dit_ctx on the current CUDA device."""
 
     def __init__(self, hidden: int, n_heads: int, head_dim: int, mlp_hidden: int, cond_dim: int,
-                 max_blocks: int, max_total_tokens: int, max_requests: int = 8, ln_eps: float = 1e-6):
+                 max_blocks: int, max_total_tokens: int, max_requests: int = 8, ln_eps: float = 1e-6,
+                 flags: int = 0):
         import torch
         self.torch = torch
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("libdit needs a CUDA device (sm_100); there is no CPU path")
         self.cfg = DitConfig(hidden, n_heads, head_dim, mlp_hidden, cond_dim, max_blocks, max_total_tokens,
-                             max_requests, ln_eps, 0)
+                             max_requests, ln_eps, flags)
         nbytes = self.lib.dit_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
             raise DitError(2, "configuration rejected by dit_workspace_bytes")
@@ -300,6 +305,19 @@ class DitContext:
                                               lens.ctypes.data_as(C.POINTER(C.c_int32)), len(lens),
                                               C.c_void_p(cond.data_ptr()), n_blocks, C.c_void_p(out.data_ptr()),
                                               self._stream(stream)))
+        return out
+
+    def dit_step_forward_requests(self, packed_tokens, reqs, cond, n_blocks: int, out=None, stream=None):
+        """dit_step_forward with the batch given as requests (needed by the rotary term)."""
+        torch = self.torch
+        assert packed_tokens.is_cuda and packed_tokens.dtype == torch.bfloat16 and packed_tokens.is_contiguous()
+        assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous()
+        assert packed_tokens.shape[1] == self.hidden and cond.shape == (len(reqs), self.cond_dim)
+        if out is None:
+            out = torch.empty(packed_tokens.shape, dtype=torch.float32, device="cuda")
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.shape == packed_tokens.shape
+        self._check(self.lib.dit_step_forward_requests(self.handle, self._ptr(packed_tokens), request_array(reqs), len(reqs),
+                                                       self._ptr(cond), n_blocks, self._ptr(out), self._stream(stream)))
         return out
 
     def dit_step_forward_host(self, host_tokens, token_lens, host_cond, n_blocks: int, host_out, stream=None):
@@ -455,9 +473,9 @@ def dit_modulation_noalloc(cond, w_ada, b_ada, mod_out, stream=None):
     return mod_out
 
 
-def context_for(dims, max_blocks: int, max_total_tokens: int, max_requests: int = 8) -> DitContext:
+def context_for(dims, max_blocks: int, max_total_tokens: int, max_requests: int = 8, flags: int = 0) -> DitContext:
     return DitContext(dims.hidden, dims.n_heads, dims.head_dim, dims.mlp_hidden, dims.cond_dim,
-                      max_blocks, max_total_tokens, max_requests, dims.ln_eps)
+                      max_blocks, max_total_tokens, max_requests, dims.ln_eps, flags)
 
 
 def upload_weights(ctx: DitContext, blocks) -> None:

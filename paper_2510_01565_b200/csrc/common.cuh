@@ -20,6 +20,14 @@ struct SeqInfo {
   int order[DIT_MAX_REQUESTS];
 };
 
+// Image geometry of the packed requests, for kernels that need a token's patch row and column:
+// the first img_cu[r+1] - img_cu[r] rows of request r are its image tokens in row-major patch order,
+// gw[r] patches per row; the rest are text tokens (position (0, 0)).
+struct RowGeom {
+  int img_cu[DIT_MAX_REQUESTS + 1];
+  int gw[DIT_MAX_REQUESTS];
+};
+
 // Device status word values (written by a kernel whose bounded wait ran out).
 enum : int { kStatusOk = 0, kStatusGemmTimeout = 1, kStatusAttnTimeout = 2 };
 

@@ -1,5 +1,6 @@
 // libdit: C ABI, context, host-side planning and kernel launches.
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -27,7 +28,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets (bytes) inside one block's weight slot.
 struct BlockLayout {
-  size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, bytes;
+  size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, q_norm, k_norm, bytes;
 };
 // Offsets (bytes) inside the workspace.
 struct Layout {
@@ -36,6 +37,7 @@ struct Layout {
   // tensors and intermediates of the shell around the block stack
   size_t sh_w_in, sh_b_in, sh_w_t1, sh_b_t1, sh_w_t2, sh_b_t2, sh_w_fa, sh_b_fa, sh_w_out, sh_b_out;
   size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok;
+  size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
   size_t bytes;
 };
 constexpr int kWoutRows = 256;   // W_out^T is stored zero-padded to one full weight tile of the GEMM
@@ -49,7 +51,7 @@ bool config_ok(const dit_config* c) {
   if (c->cond_dim < 1 || c->cond_dim > kMaxCondDim) return false;
   if (c->max_blocks < 1 || c->max_total_tokens < 1) return false;
   if (c->max_requests < 1 || c->max_requests > DIT_MAX_REQUESTS) return false;
-  if (!(c->ln_eps >= 0.f) || c->flags != 0) return false;
+  if (!(c->ln_eps >= 0.f) || (c->flags & ~static_cast<uint32_t>(DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D))) return false;
   return true;
 }
 
@@ -68,6 +70,8 @@ Layout make_layout(const dit_config& c) {
   L.blk.b_fc1 = take(F * 4);
   L.blk.w_fc2 = take(H * F * 2);
   L.blk.b_fc2 = take(H * 4);
+  L.blk.q_norm = take(c.head_dim * 4);
+  L.blk.k_norm = take(c.head_dim * 4);
   L.blk.bytes = o;
   o = 0;
   L.weights = take(L.blk.bytes * c.max_blocks);
@@ -96,6 +100,7 @@ Layout make_layout(const dit_config& c) {
   L.sh_cond = take(R * C * 2);
   L.sh_modfin = take(R * 2 * H * 4);
   L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
+  L.rope_theta = take(64 * 4);
   L.bytes = o;
   return L;
 }
@@ -169,9 +174,11 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
   return true;
 }
 
-template <int EPI>
+const RowGeom kNoGeom{};
+
+template <int EPI, int HD = 0>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
-                        const SeqInfo& seq, cudaStream_t st) {
+                        const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom) {
   // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
   GemmParams q = p;
   const long long band_bytes = 2ll * gemm_cfg::BM * p.K * 2;
@@ -179,7 +186,7 @@ cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtens
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);
-  gemm_tcgen05_kernel<EPI><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, q, seq);
+  gemm_tcgen05_kernel<EPI, HD><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, q, seq, geo);
   return cudaGetLastError();
 }
 
@@ -206,11 +213,15 @@ size_t mod_smem_bytes(int C) {   // activations [G][C], later reused for the sli
   return std::max<size_t>(static_cast<size_t>(kModReqGroup) * C, static_cast<size_t>(kModSlices) * kModReqGroup * kModCols) * sizeof(float);
 }
 
+// `geo` (image geometry of the requests) is needed by the rotary term only; NULL otherwise.
 dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
-                     float* out, cudaStream_t st) {
+                     float* out, cudaStream_t st, const RowGeom* geo = nullptr) {
   const dit_config& c = ctx->cfg;
   SeqInfo seq{};
   if (!build_seq(lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
+  const bool qk_variant = (c.flags & (DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D)) != 0;
+  if ((c.flags & DIT_FLAG_ROPE_2D) && !geo)
+    return fail(ctx, DIT_ERR_INVALID_ARG, "the rotary term needs the requests' geometry: use dit_step_forward_requests");
   const int T = seq.total, H = c.hidden, F = c.mlp_hidden;
   if (T > c.max_total_tokens) return fail(ctx, DIT_ERR_CAPACITY, "packed batch exceeds max_total_tokens");
   for (int b = 0; b < n_blocks; ++b)
@@ -283,7 +294,21 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.M = T; g.N = 3 * H; g.K = H;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_qkv);
     g.out16 = qkv;
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] { return launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st); }));
+    if (qk_variant) {
+      g.hidden = H; g.eps = c.ln_eps;
+      if (c.flags & DIT_FLAG_QK_RMSNORM) {
+        g.q_norm = reinterpret_cast<const float*>(wb + ctx->lay.blk.q_norm);
+        g.k_norm = reinterpret_cast<const float*>(wb + ctx->lay.blk.k_norm);
+      }
+      if (c.flags & DIT_FLAG_ROPE_2D) g.rope_theta = ctx->at<float>(ctx->lay.rope_theta);
+      const RowGeom& rg = geo ? *geo : kNoGeom;
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+        return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg)
+                                 : launch_gemm<kEpiQkvF16, 64>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg);
+      }));
+    } else {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] { return launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st); }));
+    }
     // attention
     AttnParams ap{};
     ap.out = a; ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
@@ -401,6 +426,8 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF32>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>), mod_smem_bytes(kMaxCondDim));  // same for every context
@@ -418,6 +445,13 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
     ctx->gemm_pairs = std::max(1, std::min(clusters, sms / 2));
   }
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
+  if (e == cudaSuccess) {
+    // rotary pair frequencies of one axis group of n = (d - d/8) / 2 channels: 10000^(-2i/n), i < n/2
+    float theta[64] = {};
+    const int n_axis = (cfg->head_dim - cfg->head_dim / 8) / 2;
+    for (int i = 0; i < n_axis / 2; ++i) theta[i] = static_cast<float>(pow(10000.0, -2.0 * i / n_axis));
+    e = cudaMemcpy(ctx->ws + lay.rope_theta, theta, sizeof(theta), cudaMemcpyHostToDevice);
+  }
   if (e != cudaSuccess) { delete[] ctx->blocks; delete ctx; return DIT_ERR_CUDA; }
   *out = ctx;
   return DIT_OK;
@@ -445,8 +479,8 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   bs.loaded = false;
 
   DIT_CUDA_TRY(ctx, cudaMemcpyAsync(base + L.w_ada, w->w_ada, static_cast<size_t>(C) * 6 * H * 2, cudaMemcpyDeviceToDevice, st));
-  auto bias = [&](const void* src, size_t off, int n) {
-    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + off), n);
+  auto bias = [&](const void* src, size_t off, int n, float fill = 0.f) {
+    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + off), n, fill);
     return cudaGetLastError();
   };
   auto weight = [&](const void* src, size_t off, int K, int N) {   // [K, N] bf16 -> [N, K] fp16
@@ -463,6 +497,8 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
   DIT_CUDA_TRY(ctx, weight(w->w_fc2, L.w_fc2, F, H));
   DIT_CUDA_TRY(ctx, bias(w->b_fc2, L.b_fc2, H));
+  DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));   // NULL scale = ones
+  DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
 
   if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) ||
       !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) ||
@@ -644,6 +680,13 @@ dit_status build_shell(dit_ctx* ctx, const dit_request* reqs, int n, const float
   return DIT_OK;
 }
 
+RowGeom geom_of(const ShellInfo& info) {
+  RowGeom g{};
+  memcpy(g.img_cu, info.img_cu, sizeof(g.img_cu));
+  memcpy(g.gw, info.gw, sizeof(g.gw));
+  return g;
+}
+
 // out[r, :] = act(in[r, :]) W + b (+ addend[r, :]): the modulation kernel with one "block".
 template <int kIn>
 cudaError_t launch_small_linear(const void* in, const void* w, const float* b, const float* addend, float* out32,
@@ -735,7 +778,7 @@ dit_status dit_load_shell_weights(dit_ctx* ctx, const dit_shell_weights* w, void
     return cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyDeviceToDevice, st);
   };
   auto bias = [&](const void* src, size_t off, int n) {
-    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), ctx->at<float>(off), n);
+    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), ctx->at<float>(off), n, 0.f);
     return cudaGetLastError();
   };
   DIT_CUDA_TRY(ctx, copy(L.sh_w_in, w->w_in, DIT_PATCH_DIM * H * 2));
@@ -811,6 +854,24 @@ dit_status dit_sampler_update(dit_ctx* ctx, float* latents, const float* velocit
   return DIT_OK;
 }
 
+dit_status dit_step_forward_requests(dit_ctx* ctx, const void* packed_tokens, const dit_request* reqs, int32_t n,
+                                     const void* cond, int32_t n_blocks, float* out, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (n < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "n_requests is negative");
+  if (n == 0) return DIT_OK;
+  if (!reqs) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  SeqInfo seq{}; ShellInfo info{};
+  dit_status s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
+  if (s != DIT_OK) return s;
+  int32_t lens[DIT_MAX_REQUESTS];
+  for (int r = 0; r < n; ++r) lens[r] = seq.cu[r + 1] - seq.cu[r];
+  s = check_step_args(ctx, packed_tokens, lens, n, cond, n_blocks, out);
+  if (s != DIT_OK) return s;
+  const RowGeom geo = geom_of(info);
+  return step_impl(ctx, packed_tokens, lens, n, cond, n_blocks, out, static_cast<cudaStream_t>(stream), &geo);
+}
+
 dit_status dit_denoise_step(dit_ctx* ctx, float* latents, const void* text_tokens, const dit_request* reqs, int32_t n,
                             const float* dsigma, const float* pooled, int32_t n_blocks, float* velocity, void* stream) {
   dit_status s = check_shell_args(ctx, reqs, n);
@@ -834,7 +895,8 @@ dit_status dit_denoise_step(dit_ctx* ctx, float* latents, const void* text_token
   if (s != DIT_OK) return s;
   s = embed_impl(ctx, latents, text_tokens, seq, info, tokens, st);
   if (s != DIT_OK) return s;
-  s = step_impl(ctx, tokens, lens, n, cond, n_blocks, x, st);       // the last block writes the residual stream in place
+  const RowGeom geo = geom_of(info);
+  s = step_impl(ctx, tokens, lens, n, cond, n_blocks, x, st, &geo);   // the last block writes the residual stream in place
   if (s != DIT_OK) return s;
   s = final_impl(ctx, x, seq, info, n, cond, velocity, latents, st);
   if (s != DIT_OK) return s;
@@ -899,7 +961,7 @@ extern "C" dit_status dit_modulation_noalloc(const void* cond, const void* w_ada
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int n6 = 6 * hidden;
   // The scratch still holds the previous call's bias: rewrite all of [0, 6H) (zeros for a NULL bias).
-  bf16_to_f32_kernel<<<(n6 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(b_ada), scratch, n6);
+  bf16_to_f32_kernel<<<(n6 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(b_ada), scratch, n6, 0.f);
   if (cudaGetLastError() != cudaSuccess) return DIT_ERR_CUDA;
   ModParams mp{};
   mp.cond = static_cast<const __nv_bfloat16*>(cond);

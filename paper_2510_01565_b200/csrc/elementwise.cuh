@@ -234,9 +234,10 @@ transpose_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __res
   }
 }
 
-__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, int n) {
+// Widens a bf16 vector to fp32; a NULL input stands for a constant vector of `fill`.
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, int n, float fill) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = in ? __bfloat162float(in[i]) : 0.f;
+  if (i < n) out[i] = in ? __bfloat162float(in[i]) : fill;
 }
 
 }  // namespace dit

@@ -18,13 +18,16 @@
 //   kEpiBiasGeluF16  out16 = gelu_tanh(acc + bias)                        (MLP up-projection)
 //   kEpiGateResidF32 out32 = resid + gate[request(row)] * (acc + bias)    (attention / MLP output)
 //   kEpiBiasF32      out32 = acc + bias                                   (output projection of the final layer)
+//   kEpiQkvF16       out16 = acc + bias, then per head of HD columns, for the Q and K thirds only:
+//                    optional RMS-norm with a learned [HD] scale and optional 2-D rotary term
+//                    (a head's columns sit in one thread, so both are thread-local)
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace dit {
 
-enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32 = 2, kEpiBiasF32 = 3 };
+enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32 = 2, kEpiBiasF32 = 3, kEpiQkvF16 = 4 };
 
 struct GemmParams {
   int M, N, K;
@@ -36,6 +39,12 @@ struct GemmParams {
   const float* gate;        // gate vector of request 0 for this block; request r at gate + r * gate_stride
   long long gate_stride;
   int* status;              // device status word
+  // kEpiQkvF16 only
+  const float* q_norm;      // [HD] RMS-norm scale of the queries, NULL = no RMS-norm
+  const float* k_norm;      // [HD] same for the keys
+  const float* rope_theta;  // [(HD - HD/8) / 4] pair frequencies of one axis group, NULL = no rotary term
+  int hidden;               // H: columns [0,H) are Q, [H,2H) K, [2H,3H) V
+  float eps;
 };
 
 namespace gemm_cfg {
@@ -68,10 +77,10 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int ban
   mb = b * band + (r - nb * rows);
 }
 
-template <int EPI>
+template <int EPI, int HD = 0>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmParams p, const __grid_constant__ SeqInfo seq) {
+                    const GemmParams p, const __grid_constant__ SeqInfo seq, const __grid_constant__ RowGeom geo) {
   using namespace gemm_cfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -190,6 +199,71 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+      if constexpr (EPI == kEpiQkvF16) {
+        // patch row and column of this lane's token (text tokens and rows past M: (0, 0))
+        int py = 0, px = 0;
+        if (p.rope_theta && row_ok) {
+          const int rq = find_request(seq, row);
+          const int local = row - seq.cu[rq];
+          if (local < geo.img_cu[rq + 1] - geo.img_cu[rq]) { py = local / geo.gw[rq]; px = local - py * geo.gw[rq]; }
+        }
+#pragma unroll 1
+        for (int hc = 0; hc < BN / HD; ++hc) {
+          const int colh = n0 + hc * HD;       // first column of this head; heads never straddle Q | K | V
+          if (colh >= p.N) break;              // warp-uniform
+          float v[HD];
+#pragma unroll
+          for (int q = 0; q < HD / 32; ++q) {
+            uint32_t r[32];
+            __syncwarp();                      // tcgen05.ld is warp-collective: reconverge first
+            tmem_ld32(t_row + hc * HD + q * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[q * 32 + i] = __uint_as_float(r[i]) + __ldg(p.bias + colh + q * 32 + i);
+          }
+          if (row_ok) {
+            const int kind = colh / p.hidden;  // 0 = Q, 1 = K, 2 = V
+            if (kind < 2) {
+              const float* g = kind == 0 ? p.q_norm : p.k_norm;
+              if (g) {
+                float ss = 0.f;
+#pragma unroll
+                for (int i = 0; i < HD; ++i) ss = fmaf(v[i], v[i], ss);
+                const float rstd = rsqrtf(ss * (1.0f / HD) + p.eps);
+#pragma unroll
+                for (int i = 0; i < HD; ++i) v[i] *= rstd * __ldg(g + i);
+              }
+              if (p.rope_theta && (py | px)) {
+                constexpr int DT = HD / 8, NA = (HD - DT) / 2;   // unrotated channels, channels per axis group
+#pragma unroll
+                for (int i = 0; i < NA / 2; ++i) {
+                  const float th = __ldg(p.rope_theta + i);
+                  float sy, cy, sx, cx;
+                  sincosf(static_cast<float>(py) * th, &sy, &cy);
+                  sincosf(static_cast<float>(px) * th, &sx, &cx);
+                  const float a = v[DT + 2 * i], b = v[DT + 2 * i + 1];
+                  v[DT + 2 * i] = a * cy - b * sy;
+                  v[DT + 2 * i + 1] = a * sy + b * cy;
+                  const float c2 = v[DT + NA + 2 * i], d2 = v[DT + NA + 2 * i + 1];
+                  v[DT + NA + 2 * i] = c2 * cx - d2 * sx;
+                  v[DT + NA + 2 * i + 1] = c2 * sx + d2 * cx;
+                }
+              }
+            }
+            uint4* dst = reinterpret_cast<uint4*>(p.out16 + static_cast<size_t>(row) * p.N + colh);
+#pragma unroll
+            for (int q = 0; q < HD / 8; ++q) {
+              uint32_t w[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const __half2 hh = __floats2half2_rn(v[8 * q + 2 * h], v[8 * q + 2 * h + 1]);
+                w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+              dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else {
 #pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
@@ -267,6 +341,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
           }
         }
+      }
       }
       tc_fence_before();
       __syncwarp();

@@ -160,6 +160,13 @@ def draw_block_weights(rng: np.random.Generator, dims: ModelDims, std: float = 0
     return {k: _normal_bf16(rng, shapes[k], std) for k in WEIGHT_NAMES}
 
 
+def draw_qk_norm(rng: np.random.Generator, dims: ModelDims) -> Dict[str, np.ndarray]:
+    """RMS-norm scales of the queries and keys, [head_dim] each, 1 + 0.1 N(0,1), bf16 bits.
+    Drawn from a generator of their own so that the ten block tensors keep their draw order."""
+    return {k: f32_to_bf16_bits(1.0 + 0.1 * rng.standard_normal(size=dims.head_dim, dtype=np.float32))
+            for k in ("q_norm", "k_norm")}
+
+
 def make_custom(name: str, dims: ModelDims, n_blocks: int,
                 reqs: Sequence[Tuple[int, int, int]], seed: int = 0,
                 timestep_cond: bool = True, with_weights: bool = True) -> Workload:

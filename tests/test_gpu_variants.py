@@ -1,0 +1,169 @@
+"""GPU parity of the model-variant parts of the block (per-head RMS-norm of queries and keys, 2-D
+rotary position term, both fused into the QKV projection's epilogue) against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import dit_oracle as O
+from oracle import step_oracle as S
+from paper_2510_01565_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-2   # max|gpu - oracle| / rms(oracle), per request
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device; the library has no CPU path")
+    from paper_2510_01565_b200 import binding, build
+    build.build_library()
+    binding.load_library()
+    return binding
+
+
+def f64w(w):
+    return {k: W.bf16_to_f64(v) for k, v in w.items()}
+
+
+def variant_workload(dims, n_blocks, reqs, seed, qk_norm):
+    wl = W.make_custom("variant", dims, n_blocks, reqs, seed=seed)
+    if qk_norm:
+        rng = np.random.default_rng(seed + 77)
+        for w in wl.weights:
+            w.update(W.draw_qk_norm(rng, dims))
+    return wl
+
+
+def oracle_out(wl, rope):
+    blocks = [f64w(w) for w in wl.weights]
+    pos = [O.patch_positions(q.height, q.width, q.n_text_tokens) for q in wl.requests] if rope else None
+    return O.step_forward(W.bf16_to_f64(wl.packed_tokens()), wl.token_lens, W.bf16_to_f64(wl.cond), blocks,
+                          wl.dims.n_heads, wl.dims.ln_eps, positions=pos)
+
+
+def run_gpu(B, wl, flags, use_requests=True):
+    import torch
+    ctx = B.context_for(wl.dims, wl.n_blocks, wl.total_tokens, len(wl.requests), flags=flags)
+    B.upload_weights(ctx, wl.weights)
+    tok, cond = B.bits_to_cuda_bf16(wl.packed_tokens()), B.bits_to_cuda_bf16(wl.cond)
+    if use_requests:
+        out = ctx.dit_step_forward_requests(tok, wl.requests, cond, wl.n_blocks)
+    else:
+        out = ctx.dit_step_forward(tok, wl.token_lens, cond, wl.n_blocks)
+    torch.cuda.synchronize()
+    ctx.dit_ctx_poll_status()
+    return ctx, out
+
+
+def check(wl, out, ref):
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    p, worst = 0, 0.0
+    for r, l in enumerate(wl.token_lens):
+        err = O.error_metric(got[p:p + l], ref[p:p + l])
+        assert err <= TOL, f"request {r}: max|d|/rms = {err:.3e}"
+        worst = max(worst, err)
+        p += l
+    return worst
+
+
+MIXED = [(64, 96, 5), (32, 32, 0), (128, 64, 17), (16, 16, 1)]
+
+
+@pytest.mark.parametrize("flags", [1, 2, 3])
+def test_small_model_head64(B, flags):
+    wl = variant_workload(W.SMALL, 2, MIXED, seed=21, qk_norm=bool(flags & 1))
+    ctx, out = run_gpu(B, wl, flags)
+    ref = oracle_out(wl, rope=bool(flags & 2))
+    check(wl, out, ref)
+    ctx.close()
+
+
+def test_qkv_tap_holds_normed_rotated_heads(B):
+    wl = variant_workload(W.SMALL, 1, MIXED, seed=22, qk_norm=True)
+    ctx, out = run_gpu(B, wl, 3)
+    got = ctx.dit_debug_tap("qkv").cpu().numpy().astype(np.float64)
+    w = f64w(wl.weights[0])
+    p = 0
+    for r, q in enumerate(wl.requests):
+        l = q.n_tokens
+        taps = {}
+        O.block_forward(W.bf16_to_f64(wl.tokens[r]), W.bf16_to_f64(wl.cond[r]), w, wl.dims.n_heads, wl.dims.ln_eps,
+                        taps=taps, positions=O.patch_positions(q.height, q.width, q.n_text_tokens))
+        assert O.error_metric(got[p:p + l], taps["qkv"]) <= TOL, f"request {r}"
+        if q.n_image_tokens > 1:
+            # the comparison has teeth: without the variants the queries and keys are far outside the bar
+            plain = {}
+            O.block_forward(W.bf16_to_f64(wl.tokens[r]), W.bf16_to_f64(wl.cond[r]),
+                            {k: v for k, v in w.items() if k not in ("q_norm", "k_norm")}, wl.dims.n_heads,
+                            wl.dims.ln_eps, taps=plain)
+            assert O.error_metric(got[p:p + l], plain["qkv"]) > 10 * TOL
+        p += l
+    ctx.close()
+
+
+def test_large_model_head128(B):
+    wl = variant_workload(W.LARGE, 1, [(256, 256, 64), (128, 256, 0)], seed=23, qk_norm=True)
+    ctx, out = run_gpu(B, wl, 3)
+    check(wl, out, oracle_out(wl, rope=True))
+    ctx.close()
+
+
+def test_packed_equals_alone_and_entry_points(B):
+    import torch
+    wl = variant_workload(W.SMALL, 2, MIXED, seed=24, qk_norm=True)
+    ctx, out = run_gpu(B, wl, 3)
+    cu = np.concatenate([[0], np.cumsum(wl.token_lens)])
+    tok, cond = B.bits_to_cuda_bf16(wl.packed_tokens()), B.bits_to_cuda_bf16(wl.cond)
+    for r in range(len(wl.requests)):
+        a, b = int(cu[r]), int(cu[r + 1])
+        alone = ctx.dit_step_forward_requests(tok[a:b].contiguous(), [wl.requests[r]], cond[r:r + 1].contiguous(), 2)
+        torch.cuda.synchronize()
+        assert torch.equal(alone, out[a:b]), f"request {r}: packed and alone outputs differ"
+    # without geometry the rotary term cannot run
+    with pytest.raises(B.DitError) as e:
+        ctx.dit_step_forward(tok, wl.token_lens, cond, 2)
+    assert e.value.status == 1
+    ctx.close()
+    # RMS-norm alone needs no geometry: both entry points agree bit for bit
+    ctx1, out1 = run_gpu(B, wl, 1, use_requests=False)
+    ctx2, out2 = run_gpu(B, wl, 1, use_requests=True)
+    assert torch.equal(out1, out2)
+    ctx1.close(); ctx2.close()
+    # a context without flags ignores q_norm / k_norm and matches the plain oracle
+    ctx0, out0 = run_gpu(B, wl, 0)
+    plain = [f64w({k: v for k, v in w.items() if k not in ("q_norm", "k_norm")}) for w in wl.weights]
+    ref = O.step_forward(W.bf16_to_f64(wl.packed_tokens()), wl.token_lens, W.bf16_to_f64(wl.cond), plain,
+                         wl.dims.n_heads, wl.dims.ln_eps)
+    check(wl, out0, ref)
+    ctx0.close()
+
+
+def test_full_denoise_step_with_variants(B):
+    import torch
+    reqs = [(64, 96, 5), (32, 32, 0), (96, 32, 2)]
+    si = W.make_step_inputs(W.SMALL, 2, reqs, seed=25)
+    rng = np.random.default_rng(99)
+    for w in si.weights:
+        w.update(W.draw_qk_norm(rng, si.dims))
+    ctx = B.context_for(si.dims, 2, sum(si.token_lens), len(reqs), flags=3)
+    B.upload_weights(ctx, si.weights)
+    B.upload_shell_weights(ctx, si.shell)
+    latents = torch.from_numpy(np.concatenate([z.reshape(-1) for z in si.latents])).cuda()
+    vel = torch.empty_like(latents)
+    text = B.bits_to_cuda_bf16(np.concatenate(si.texts, axis=0))
+    ctx.dit_denoise_step(latents, text, si.requests, si.dsigmas, torch.from_numpy(si.pooled).cuda(), 2, velocity=vel)
+    torch.cuda.synchronize()
+    ctx.dit_ctx_poll_status()
+    _, vels, _ = S.denoise_step([z.astype(np.float64) for z in si.latents], [W.bf16_to_f64(t) for t in si.texts],
+                                [q.timestep for q in si.requests], [float(d) for d in si.dsigmas],
+                                [p.astype(np.float64) for p in si.pooled], f64w(si.shell), [f64w(w) for w in si.weights],
+                                si.dims.n_heads, si.dims.ln_eps, rope=True)
+    got, p = vel.cpu().numpy().astype(np.float64), 0
+    for r, v in enumerate(vels):
+        err = O.error_metric(got[p:p + v.size].reshape(v.shape), v)
+        assert err <= TOL, f"request {r}: {err:.3e}"
+        p += v.size
+    ctx.close()
