@@ -179,13 +179,21 @@ def run_gpu(args):
         nb = args.depth
         wl.weights = [wl.weights[b % len(wl.weights)] for b in range(nb)]
         wl.n_blocks = nb
-    ctx = B.context_for(wl.dims, nb, wl.total_tokens, len(wl.requests))
+    if args.variants & 1:
+        qk_rng = np.random.default_rng(args.seed + 2000)
+        wl.weights = [dict(w, **W.draw_qk_norm(qk_rng, wl.dims)) for w in wl.weights]
+    ctx = B.context_for(wl.dims, nb, wl.total_tokens, len(wl.requests), flags=args.variants)
     B.upload_weights(ctx, wl.weights)
     lens = wl.token_lens
     tok_bits, cond_bits = wl.packed_tokens(), wl.cond
     tok, cond = B.bits_to_cuda_bf16(tok_bits), B.bits_to_cuda_bf16(cond_bits)
     out = torch.empty((wl.total_tokens, wl.dims.hidden), dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
+    if args.variants:
+        # the rotary term needs each token's patch position: the step is given the requests themselves
+        step = lambda: ctx.dit_step_forward_requests(tok, wl.requests, cond, nb, out=out)
+    else:
+        step = lambda: ctx.dit_step_forward(tok, lens, cond, nb, out=out)
 
     def barrier():
         if dist is not None:
@@ -197,7 +205,7 @@ def run_gpu(args):
 
     # ---------------------------------------------------------------- device-resident throughput
     for _ in range(args.warmup):
-        ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+        step()
     barrier()
     ctx.dit_ctx_poll_status()
     sampler = ClockSampler(local_rank)
@@ -207,7 +215,7 @@ def run_gpu(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+        step()
     e1.record(stream)
     barrier()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
@@ -230,12 +238,12 @@ def run_gpu(args):
         side = torch.cuda.Stream()
         side.wait_stream(stream)
         with torch.cuda.stream(side):
-            ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+            step()
         stream.wait_stream(side)
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+            step()
         for _ in range(args.warmup):
             g.replay()
         barrier()
@@ -253,11 +261,22 @@ def run_gpu(args):
     h_cond = torch.from_numpy(cond_bits.view(np.int16)).pin_memory()
     h_out = torch.empty((wl.total_tokens, wl.dims.hidden), dtype=torch.float32).pin_memory()
     e2e_steps = max(1, min(args.steps, 5))
-    ctx.dit_step_forward_host(h_tok, lens, h_cond, nb, h_out)
+
+    def e2e_step():
+        if args.variants & 2:     # the host-buffer entry point carries no geometry: copy, run, copy back by hand
+            tok.copy_(h_tok.view(torch.bfloat16), non_blocking=True)
+            cond.copy_(h_cond.view(torch.bfloat16), non_blocking=True)
+            step()
+            h_out.copy_(out, non_blocking=True)
+            stream.synchronize()
+        else:
+            ctx.dit_step_forward_host(h_tok, lens, h_cond, nb, h_out)
+
+    e2e_step()
     barrier()
     e0.record(stream)
     for _ in range(e2e_steps):
-        ctx.dit_step_forward_host(h_tok, lens, h_cond, nb, h_out)
+        e2e_step()
     e1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
@@ -348,7 +367,7 @@ def run_gpu(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
-            "config": {"workload": wl.name, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
+            "config": {"workload": wl.name, "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2)}, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
                        "total_tokens": T, "image_tokens": wl.image_tokens, "hidden": H, "heads": wl.dims.n_heads,
                        "head_dim": wl.dims.head_dim, "mlp_hidden": F, "parallelism": f"replicas x{world}",
                        "l2": "weights and activations of a step exceed L2 (126 MB); no flush"},
@@ -376,6 +395,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0, help="run this many blocks instead of the configuration's (weights reused cyclically)")
+    ap.add_argument("--variants", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="block variant bits: 1 = RMS-norm of queries and keys, 2 = 2-D rotary term (not the headline configuration)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
