@@ -30,6 +30,10 @@ FLUX / SD3 class models): per-head RMS-norm of queries and keys with a learned
 channels of a head unrotated, then a patch-row group and a patch-column group
 of equal size, adjacent channel pairs, base 10000; text tokens at (0, 0)).
 
+A second block form, `parallel_block_forward`: one modulation triple, attention
+and MLP both read the same modulated LayerNorm output, one output projection
+over their concatenation (the "single-stream" blocks of the FLUX family).
+
 Every function works on fp64 arrays.  Nothing is tiled, fused or reordered
 beyond taking query rows in slabs to bound memory (each softmax row is still
 the full definition over all keys of the request).
@@ -218,11 +222,48 @@ def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps
     return y
 
 
+def parallel_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps: float,
+                           rows: np.ndarray | None = None, taps: dict | None = None,
+                           positions: np.ndarray | None = None) -> np.ndarray:
+    """The parallel (single-modulation) form of the block: attention and the MLP read the same
+    modulated LayerNorm output, their results are concatenated and share one output projection:
+
+        (shift, scale, gate) = SiLU(cond) W_ada + b_ada                    W_ada [C, 3H]
+        h = LN(x) (1 + scale) + shift
+        a = attention(h W_qkv + b_qkv),   u = gelu_tanh(h W_fc1 + b_fc1)
+        y = x + gate * ([a | u] W_out + b_out)                             W_out [H + F, H]
+
+    Optional q_norm / k_norm and `positions` act on queries and keys as in block_forward.
+    """
+    H = x.shape[1]
+    shift, scale, gate = np.split(silu(cond) @ w["w_ada"] + w["b_ada"], 3)
+    h = modulate(layer_norm(x, eps), shift, scale)
+    qkv = h @ w["w_qkv"] + w["b_qkv"]
+    q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+    if "q_norm" in w:
+        q = rms_norm_heads(q, w["q_norm"], n_heads, eps)
+        k = rms_norm_heads(k, w["k_norm"], n_heads, eps)
+    if positions is not None:
+        q, k = rope_2d(q, positions, n_heads), rope_2d(k, positions, n_heads)
+    a = attention(q, k, v, n_heads, rows)
+    hr, xr = (h, x) if rows is None else (h[rows], x[rows])
+    u = gelu_tanh(hr @ w["w_fc1"] + w["b_fc1"])
+    y = xr + gate * (np.concatenate([a, u], axis=1) @ w["w_out"] + w["b_out"])
+    if taps is not None:
+        taps.update(h1=h, qkv=np.concatenate([q, k, v], axis=1), a=a, u=u)
+    return y
+
+
+def any_block_forward(x, cond, w: Weights, n_heads: int, eps: float, **kw) -> np.ndarray:
+    """Dispatch on the block's form: a parallel block is the one that holds "w_out"."""
+    return (parallel_block_forward if "w_out" in w else block_forward)(x, cond, w, n_heads, eps, **kw)
+
+
 def stack_forward_alone(x: np.ndarray, cond: np.ndarray, blocks: Sequence[Weights],
                         n_heads: int, eps: float, positions: np.ndarray | None = None) -> np.ndarray:
     """A stack of blocks on one request run by itself."""
     for w in blocks:
-        x = block_forward(x, cond, w, n_heads, eps, positions=positions)
+        x = any_block_forward(x, cond, w, n_heads, eps, positions=positions)
     return x
 
 

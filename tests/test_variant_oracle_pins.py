@@ -129,3 +129,64 @@ def test_taps_hold_normed_and_rotated_queries():
     want_q = O.rope_2d(O.rms_norm_heads(raw[:, :H], w["q_norm"], heads, 1e-6), pos, heads)
     assert np.array_equal(taps["qkv"][:, :H], want_q)
     assert np.array_equal(taps["qkv"][:, 2 * H:], raw[:, 2 * H:])      # values are neither normed nor rotated
+
+
+# ----------------------------------------------------------------------------- the parallel block form
+def test_parallel_block_reduces_to_halves_of_the_sequential_block():
+    rng = np.random.default_rng(7)
+    H, F, C, heads, L = 64, 128, 8, 2, 5
+    w = _block(rng, H, F, C)
+    w["b_o"] = rng.standard_normal(H) * 0.1
+    w["b_fc2"] = rng.standard_normal(H) * 0.1
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    sh_a, sc_a, g_a, sh_m, sc_m, g_m = np.split(w["w_ada"], 6, axis=1)
+    bsh_a, bsc_a, bg_a, bsh_m, bsc_m, bg_m = np.split(w["b_ada"], 6)
+    zero_w, zero_b = np.zeros_like(g_a), np.zeros_like(bg_a)
+
+    # (1) attention half: the parallel block whose output projection ignores the MLP columns equals the
+    #     sequential block with a zero MLP gate
+    par = {"w_ada": np.concatenate([sh_a, sc_a, g_a], axis=1), "b_ada": np.concatenate([bsh_a, bsc_a, bg_a]),
+           "w_qkv": w["w_qkv"], "b_qkv": w["b_qkv"], "w_fc1": w["w_fc1"], "b_fc1": w["b_fc1"],
+           "w_out": np.concatenate([w["w_o"], np.zeros((F, H))], axis=0), "b_out": w["b_o"]}
+    seq = dict(w, w_ada=np.concatenate([sh_a, sc_a, g_a, sh_m, sc_m, zero_w], axis=1),
+               b_ada=np.concatenate([bsh_a, bsc_a, bg_a, bsh_m, bsc_m, zero_b]))
+    assert np.allclose(O.parallel_block_forward(x, cond, par, heads, 1e-6), O.block_forward(x, cond, seq, heads, 1e-6), atol=1e-13)
+
+    # (2) MLP half: ignoring the attention columns equals the sequential block with a zero attention
+    #     gate, whose second LayerNorm then sees x itself
+    par2 = dict(par, w_ada=np.concatenate([sh_m, sc_m, g_m], axis=1), b_ada=np.concatenate([bsh_m, bsc_m, bg_m]),
+                w_out=np.concatenate([np.zeros((H, H)), w["w_fc2"]], axis=0), b_out=w["b_fc2"])
+    seq2 = dict(w, w_ada=np.concatenate([sh_a, sc_a, zero_w, sh_m, sc_m, g_m], axis=1),
+                b_ada=np.concatenate([bsh_a, bsc_a, zero_b, bsh_m, bsc_m, bg_m]))
+    assert np.allclose(O.parallel_block_forward(x, cond, par2, heads, 1e-6), O.block_forward(x, cond, seq2, heads, 1e-6), atol=1e-13)
+
+    # (3) the two halves add up: with one modulation triple, full = x + (attention half - x) + (MLP half - x)
+    tri_w, tri_b = np.concatenate([sh_a, sc_a, g_a], axis=1), np.concatenate([bsh_a, bsc_a, bg_a])
+    full = dict(par, w_ada=tri_w, b_ada=tri_b, w_out=np.concatenate([w["w_o"], w["w_fc2"]], axis=0), b_out=w["b_o"] + w["b_fc2"])
+    half_a = dict(full, w_out=np.concatenate([w["w_o"], np.zeros((F, H))], axis=0), b_out=w["b_o"])
+    half_m = dict(full, w_out=np.concatenate([np.zeros((H, H)), w["w_fc2"]], axis=0), b_out=w["b_fc2"])
+    ya, ym = (O.parallel_block_forward(x, cond, ww, heads, 1e-6) for ww in (half_a, half_m))
+    assert np.allclose(O.parallel_block_forward(x, cond, full, heads, 1e-6), ya + ym - x, atol=1e-13)
+
+
+def test_parallel_block_zero_gate_rows_and_dispatch():
+    rng = np.random.default_rng(8)
+    H, F, C, heads, L = 64, 128, 8, 2, 6
+    par = {"w_ada": rng.standard_normal((C, 3 * H)) * 0.1, "b_ada": rng.standard_normal(3 * H) * 0.1,
+           "w_qkv": rng.standard_normal((H, 3 * H)) * 0.2, "b_qkv": rng.standard_normal(3 * H) * 0.1,
+           "w_fc1": rng.standard_normal((H, F)) * 0.2, "b_fc1": rng.standard_normal(F) * 0.1,
+           "w_out": rng.standard_normal((H + F, H)) * 0.2, "b_out": rng.standard_normal(H) * 0.1}
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    y = O.parallel_block_forward(x, cond, par, heads, 1e-6)
+    # zero gate: identity
+    z = dict(par, w_ada=par["w_ada"].copy(), b_ada=par["b_ada"].copy())
+    z["w_ada"][:, 2 * H:] = 0.0
+    z["b_ada"][2 * H:] = 0.0
+    assert np.array_equal(O.parallel_block_forward(x, cond, z, heads, 1e-6), x)
+    # row subset == the same rows of the full result
+    rows = np.array([4, 1])
+    assert np.allclose(O.parallel_block_forward(x, cond, par, heads, 1e-6, rows=rows), y[rows], atol=1e-14)
+    # a stack mixes the two forms by what each block holds
+    seq = _block(rng, H, F, C)
+    want = O.parallel_block_forward(O.block_forward(x, cond, seq, heads, 1e-6), cond, par, heads, 1e-6)
+    assert np.array_equal(O.stack_forward_alone(x, cond, [seq, par], heads, 1e-6), want)
