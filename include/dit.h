@@ -122,6 +122,23 @@ dit_status dit_ctx_destroy(dit_ctx *ctx);
  * caller's tensors may be freed once the stream has passed this point. */
 dit_status dit_load_block_weights(dit_ctx *ctx, int32_t block_idx, const dit_block_weights *w, void *stream);
 
+/* The parallel form of the block (the single-stream blocks of the FLUX family the paper serves):
+ * one modulation triple, attention and MLP read the same modulated LayerNorm output, and one output
+ * projection runs over their concatenation:
+ *   (shift, scale, gate) = W_ada^T SiLU(c) + b_ada;   h = LN(x)(1 + scale) + shift
+ *   a = attention(h W_qkv + b_qkv);  u = gelu_tanh(h W_fc1 + b_fc1);  x = x + gate * ([a | u] W_out + b_out)
+ * Device pointers, bf16, row-major [in, out]; a NULL bias means zero, NULL q_norm / k_norm mean ones.
+ *   w_ada [C, 3H]  b_ada [3H]   w_qkv [H, 3H]  b_qkv [3H]   w_fc1 [H, F]  b_fc1 [F]
+ *   w_out [H + F, H] (attention rows first)  b_out [H]      q_norm [d]  k_norm [d]
+ * A stack may mix both forms block by block; a block slot holds whichever form was loaded last.
+ * The step runs 5 kernels for such a block instead of 7 (the attention kernel and the up-projection
+ * write side by side into one [T, H + F] buffer, so the concatenation costs nothing). */
+typedef struct {
+  const void *w_ada, *b_ada, *w_qkv, *b_qkv, *w_fc1, *b_fc1, *w_out, *b_out, *q_norm, *k_norm;
+} dit_parallel_block_weights;
+dit_status dit_load_parallel_block_weights(dit_ctx *ctx, int32_t block_idx, const dit_parallel_block_weights *w,
+                                           void *stream);
+
 /* Packer, host only, integer only (Section 6.1 token rule; requests keep their input order; inside
  * a request image tokens come first, then text tokens).  All arrays are HOST memory owned by the
  * caller: token_lens [n], cu_seqlens [n+1], row_req / row_local [sum of lens] (either may be NULL).

@@ -23,7 +23,7 @@ STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPAC
 KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
-EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights",
+EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
            "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
@@ -44,6 +44,11 @@ class DitRequest(C.Structure):
 class DitBlockWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_o", "b_o",
                                           "w_fc1", "b_fc1", "w_fc2", "b_fc2", "q_norm", "k_norm")]
+
+
+class DitParallelBlockWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_fc1", "b_fc1", "w_out", "b_out",
+                                          "q_norm", "k_norm")]
 
 
 class DitShellWeights(C.Structure):
@@ -91,6 +96,8 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_destroy.argtypes = [vp]
     lib.dit_load_block_weights.restype = C.c_int
     lib.dit_load_block_weights.argtypes = [vp, i32, C.POINTER(DitBlockWeights), vp]
+    lib.dit_load_parallel_block_weights.restype = C.c_int
+    lib.dit_load_parallel_block_weights.argtypes = [vp, i32, C.POINTER(DitParallelBlockWeights), vp]
     lib.dit_pack_requests.restype = C.c_int
     lib.dit_pack_requests.argtypes = [C.POINTER(DitRequest), i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32),
                                       C.POINTER(i32), C.POINTER(i32)]
@@ -278,6 +285,18 @@ class DitContext:
             keep.append(t)
             setattr(w, name, t.data_ptr())
         self._check(self.lib.dit_load_block_weights(self.handle, block_idx, C.byref(w), self._stream(stream)))
+
+    def dit_load_parallel_block_weights(self, block_idx: int, weights: Dict[str, "object"], stream=None):
+        """Parallel-form block: name -> CUDA bf16 tensor ([in, out] row-major); biases and norms may be None."""
+        w = DitParallelBlockWeights()
+        keep = []
+        for name, _ in DitParallelBlockWeights._fields_:
+            t = weights.get(name)
+            if t is not None:
+                assert t.is_cuda and t.dtype == self.torch.bfloat16 and t.is_contiguous(), name
+                keep.append(t)
+            setattr(w, name, t.data_ptr() if t is not None else None)
+        self._check(self.lib.dit_load_parallel_block_weights(self.handle, block_idx, C.byref(w), self._stream(stream)))
 
     def dit_pack_tokens(self, per_request_tokens: List["object"], stream=None):
         torch = self.torch
@@ -483,7 +502,10 @@ def upload_weights(ctx: DitContext, blocks) -> None:
     import torch
     for b, w in enumerate(blocks):
         dev = {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in w.items()}
-        ctx.dit_load_block_weights(b, dev)
+        if "w_out" in w:          # the parallel form of the block
+            ctx.dit_load_parallel_block_weights(b, dev)
+        else:
+            ctx.dit_load_block_weights(b, dev)
         torch.cuda.synchronize()
         del dev
 

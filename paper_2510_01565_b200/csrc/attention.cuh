@@ -28,7 +28,8 @@
 namespace dit {
 
 struct AttnParams {
-  __half* out;        // [T, H]
+  __half* out;        // [T, H] with row stride ld_out (elements)
+  int ld_out;
   int H;
   int n_heads;
   float scale_log2;   // log2(e) / sqrt(d)
@@ -278,7 +279,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       tc_fence_after();
       const float inv = 1.0f / l;
       const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
-      __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.H + head * D;
+      __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.ld_out + head * D;
 #pragma unroll 1
       for (int ch = 0; ch < D / 32; ++ch) {
         uint32_t r[32];

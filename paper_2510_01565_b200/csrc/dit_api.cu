@@ -64,10 +64,12 @@ Layout make_layout(const dit_config& c) {
   L.blk.b_ada = take(6 * H * 4);
   L.blk.w_qkv = take(3 * H * H * 2);
   L.blk.b_qkv = take(3 * H * 4);
-  L.blk.w_o = take(H * H * 2);
   L.blk.b_o = take(H * 4);
   L.blk.w_fc1 = take(F * H * 2);
   L.blk.b_fc1 = take(F * 4);
+  // W_o and W_fc2 are neighbours with no gap (H * H * 2 is a multiple of the alignment): a parallel
+  // block stores its single output projection [H, H + F] over both
+  L.blk.w_o = take(H * H * 2);
   L.blk.w_fc2 = take(H * F * 2);
   L.blk.b_fc2 = take(H * 4);
   L.blk.q_norm = take(c.head_dim * 4);
@@ -107,6 +109,7 @@ Layout make_layout(const dit_config& c) {
 
 struct BlockState {
   bool loaded = false;
+  bool parallel = false;                   // parallel form: tm_o is unused, tm_fc2 maps W_out^T [H, H + F]
   CUtensorMap tm_qkv, tm_o, tm_fc1, tm_fc2;
 };
 
@@ -124,6 +127,7 @@ struct dit_ctx {
   CUtensorMap tm_wout;                     // W_out^T, fp16 [kWoutRows, H]
   int64_t last_launches;
   int last_T, last_R, last_nb;
+  bool last_parallel;                      // the last block of the last step was a parallel block
   char err[256];
   // optional per-kernel timing (CUDA events recorded around every launch of a step)
   bool timing;
@@ -235,9 +239,13 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   float* mod = ctx->at<float>(ctx->lay.mod);
   int* status = ctx->at<int>(ctx->lay.status);
 
-  CUtensorMap tm_h, tm_a, tm_u, tm_qkv;
+  // a parallel block writes attention and MLP outputs side by side into one [T, H + F] buffer that
+  // starts where `a` starts and runs on into `u` (the two regions are consecutive)
+  __half* cat = a;
+  CUtensorMap tm_h, tm_a, tm_u, tm_qkv, tm_cat;
   if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM) || !make_map(ctx, &tm_a, a, H, T, gemm_cfg::BM) ||
-      !make_map(ctx, &tm_u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &tm_qkv, qkv, 3 * H, T, 128))
+      !make_map(ctx, &tm_u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &tm_qkv, qkv, 3 * H, T, 128) ||
+      !make_map(ctx, &tm_cat, cat, H + F, T, gemm_cfg::BM))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
 
   int64_t launches = 0;
@@ -311,7 +319,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }
     // attention
     AttnParams ap{};
-    ap.out = a; ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
+    ap.out = bs.parallel ? cat : a; ap.ld_out = bs.parallel ? H + F : H;
+    ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
 #ifdef DIT_ATTN_TRACE
     { const char* e_ = getenv("DIT_TRACE_PTR"); ap.trace = e_ ? reinterpret_cast<long long*>(strtoull(e_, nullptr, 0)) : nullptr; }
 #endif
@@ -319,6 +328,24 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_ATTENTION, [&] {
       return c.head_dim == 128 ? launch_attention<128>(tm_qkv, ap, seq, st) : launch_attention<64>(tm_qkv, ap, seq, st);
     }));
+    if (bs.parallel) {
+      // MLP up-projection + GELU-tanh from the same h, written beside the attention output
+      g = GemmParams{};
+      g.status = status;
+      g.M = T; g.N = F; g.K = H;
+      g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
+      g.out16 = cat + H; g.ld16 = H + F;
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st); }));
+      // one output projection over [attention | MLP] + gate + residual
+      g = GemmParams{};
+      g.status = status;
+      g.M = T; g.N = H; g.K = H + F;
+      g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
+      g.resid = stream; g.out32 = (b == n_blocks - 1) ? out : stream;
+      g.gate = modb + 2 * H; g.gate_stride = req_stride;
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
+      continue;
+    }
     // output projection + gate + residual
     g = GemmParams{};
     g.status = status;
@@ -349,6 +376,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   }
   ctx->last_launches = launches;
   ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
+  ctx->last_parallel = ctx->blocks[n_blocks - 1].parallel;
   return DIT_OK;
 }
 
@@ -413,6 +441,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->shell_loaded = false;
   ctx->last_launches = 0;
   ctx->last_T = ctx->last_R = ctx->last_nb = 0;
+  ctx->last_parallel = false;
   ctx->timing = false;
   ctx->ev_used = 0;
   ctx->err[0] = 0;
@@ -477,6 +506,7 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   const BlockLayout& L = ctx->lay.blk;
   BlockState& bs = ctx->blocks[b];
   bs.loaded = false;
+  bs.parallel = false;
 
   DIT_CUDA_TRY(ctx, cudaMemcpyAsync(base + L.w_ada, w->w_ada, static_cast<size_t>(C) * 6 * H * 2, cudaMemcpyDeviceToDevice, st));
   auto bias = [&](const void* src, size_t off, int n, float fill = 0.f) {
@@ -504,6 +534,52 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
       !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) ||
       !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) ||
       !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+  bs.loaded = true;
+  return DIT_OK;
+}
+
+dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_parallel_block_weights* w, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (!w) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weights");
+  if (b < 0 || b >= ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "block index outside [0, max_blocks)");
+  if (!w->w_ada || !w->w_qkv || !w->w_fc1 || !w->w_out) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL weight matrix");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int H = ctx->cfg.hidden, F = ctx->cfg.mlp_hidden, C = ctx->cfg.cond_dim;
+  uint8_t* base = ctx->block_base(b);
+  const BlockLayout& L = ctx->lay.blk;
+  BlockState& bs = ctx->blocks[b];
+  bs.loaded = false;
+  bs.parallel = true;
+
+  // The modulation kernel produces six H-wide vectors per block for the whole stack in one launch; a
+  // parallel block has three (shift, scale, gate): its W_ada / b_ada fill the first three, the rest is zero.
+  DIT_CUDA_TRY(ctx, cudaMemsetAsync(base + L.w_ada, 0, static_cast<size_t>(C) * 6 * H * 2, st));
+  DIT_CUDA_TRY(ctx, cudaMemcpy2DAsync(base + L.w_ada, static_cast<size_t>(6) * H * 2, w->w_ada, static_cast<size_t>(3) * H * 2,
+                                      static_cast<size_t>(3) * H * 2, C, cudaMemcpyDeviceToDevice, st));
+  auto bias = [&](const void* src, size_t off, int n, float fill = 0.f) {
+    bf16_to_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + off), n, fill);
+    return cudaGetLastError();
+  };
+  auto weight = [&](const void* src, size_t off, int K, int N) {   // [K, N] bf16 -> [N, K] fp16
+    dim3 grid((N + 31) / 32, (K + 31) / 32);
+    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    return cudaGetLastError();
+  };
+  DIT_CUDA_TRY(ctx, cudaMemsetAsync(base + L.b_ada, 0, static_cast<size_t>(6) * H * 4, st));
+  DIT_CUDA_TRY(ctx, bias(w->b_ada, L.b_ada, 3 * H));
+  DIT_CUDA_TRY(ctx, weight(w->w_qkv, L.w_qkv, H, 3 * H));
+  DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
+  DIT_CUDA_TRY(ctx, weight(w->w_fc1, L.w_fc1, H, F));
+  DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
+  DIT_CUDA_TRY(ctx, weight(w->w_out, L.w_o, H + F, H));          // runs on over the W_fc2 region
+  DIT_CUDA_TRY(ctx, bias(w->b_out, L.b_fc2, H));
+  DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));
+  DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
+  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) ||
+      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) ||
+      !make_map(ctx, &bs.tm_fc2, base + L.w_o, H + F, H, gemm_cfg::BN / 2))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;
   return DIT_OK;
@@ -599,6 +675,8 @@ dit_status dit_ctx_poll_status(dit_ctx* ctx) {
 dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t* rows, int64_t* cols, int32_t* elem_bytes) {
   if (!ctx || !ptr || !rows || !cols || !elem_bytes) return DIT_ERR_INVALID_ARG;
   const int64_t H = ctx->cfg.hidden, F = ctx->cfg.mlp_hidden, T = ctx->last_T;
+  if (ctx->last_parallel && (which == DIT_TAP_ATTN || which == DIT_TAP_U))
+    return fail(ctx, DIT_ERR_INVALID_ARG, "a parallel block keeps attention and MLP outputs interleaved: no dense tap");
   switch (which) {
     case DIT_TAP_H: *ptr = ctx->ws + ctx->lay.h; *rows = T; *cols = H; *elem_bytes = 2; break;
     case DIT_TAP_QKV: *ptr = ctx->ws + ctx->lay.qkv; *rows = T; *cols = 3 * H; *elem_bytes = 2; break;

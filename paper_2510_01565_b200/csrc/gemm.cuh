@@ -33,11 +33,12 @@ struct GemmParams {
   int M, N, K;
   int band;                 // row tiles (of 256 rows) per band of the tile order, >= 1
   const float* bias;        // [N]
-  __half* out16;            // [M, N]
+  __half* out16;            // [M, N] with row stride ld16 elements (0 = N)
   const float* resid;       // [M, N]
   float* out32;             // [M, N]
   const float* gate;        // gate vector of request 0 for this block; request r at gate + r * gate_stride
   long long gate_stride;
+  int ld16;
   int* status;              // device status word
   // kEpiQkvF16 only
   const float* q_norm;      // [HD] RMS-norm scale of the queries, NULL = no RMS-norm
@@ -316,7 +317,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           __syncwarp();                        // staging buffer is reused by the next chunk
         } else if (row_ok) {
           const bool full = (col0 + 32 <= p.N);
-          __half* dst = p.out16 + static_cast<size_t>(row) * p.N + col0;
+          __half* dst = p.out16 + static_cast<size_t>(row) * (p.ld16 ? p.ld16 : p.N) + col0;
           if (full) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {

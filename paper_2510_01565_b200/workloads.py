@@ -160,6 +160,17 @@ def draw_block_weights(rng: np.random.Generator, dims: ModelDims, std: float = 0
     return {k: _normal_bf16(rng, shapes[k], std) for k in WEIGHT_NAMES}
 
 
+PARALLEL_WEIGHT_NAMES = ("w_ada", "b_ada", "w_qkv", "b_qkv", "w_fc1", "b_fc1", "w_out", "b_out")
+
+
+def draw_parallel_block_weights(rng: np.random.Generator, dims: ModelDims, std: float = 0.02) -> Dict[str, np.ndarray]:
+    """One parallel-form block's eight tensors, row-major [in, out], bf16 bits, fixed draw order."""
+    h, f, c = dims.hidden, dims.mlp_hidden, dims.cond_dim
+    shapes = {"w_ada": (c, 3 * h), "b_ada": (3 * h,), "w_qkv": (h, 3 * h), "b_qkv": (3 * h,),
+              "w_fc1": (h, f), "b_fc1": (f,), "w_out": (h + f, h), "b_out": (h,)}
+    return {k: _normal_bf16(rng, shapes[k], std) for k in PARALLEL_WEIGHT_NAMES}
+
+
 def draw_qk_norm(rng: np.random.Generator, dims: ModelDims) -> Dict[str, np.ndarray]:
     """RMS-norm scales of the queries and keys, [head_dim] each, 1 + 0.1 N(0,1), bf16 bits.
     Drawn from a generator of their own so that the ten block tensors keep their draw order."""

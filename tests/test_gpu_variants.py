@@ -167,3 +167,56 @@ def test_full_denoise_step_with_variants(B):
         assert err <= TOL, f"request {r}: {err:.3e}"
         p += v.size
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- the parallel block form
+def mixed_stack_workload(dims, kinds, reqs, seed, qk_norm):
+    """kinds: string of 's' (sequential) / 'p' (parallel) per block."""
+    wl = W.make_custom("stack", dims, len(kinds), reqs, seed=seed)
+    rng = np.random.default_rng(seed + 500)
+    for b, kind in enumerate(kinds):
+        if kind == "p":
+            wl.weights[b] = W.draw_parallel_block_weights(rng, dims)
+        if qk_norm:
+            wl.weights[b].update(W.draw_qk_norm(rng, dims))
+    return wl
+
+
+@pytest.mark.parametrize("flags", [0, 3])
+def test_parallel_blocks_in_a_mixed_stack(B, flags):
+    import torch
+    wl = mixed_stack_workload(W.SMALL, "spp", MIXED, seed=31, qk_norm=bool(flags & 1))
+    ctx, out = run_gpu(B, wl, flags)
+    assert ctx.dit_last_launch_count() == 1 + 7 + 5 + 5
+    check(wl, out, oracle_out(wl, rope=bool(flags & 2)))
+    # packed == alone, bit for bit
+    cu = np.concatenate([[0], np.cumsum(wl.token_lens)])
+    tok, cond = B.bits_to_cuda_bf16(wl.packed_tokens()), B.bits_to_cuda_bf16(wl.cond)
+    for r in (0, 2):
+        a, b = int(cu[r]), int(cu[r + 1])
+        alone = ctx.dit_step_forward_requests(tok[a:b].contiguous(), [wl.requests[r]], cond[r:r + 1].contiguous(), 3)
+        torch.cuda.synchronize()
+        assert torch.equal(alone, out[a:b]), f"request {r}"
+    # the dense attention / MLP taps do not exist after a parallel block
+    with pytest.raises(B.DitError):
+        ctx.dit_debug_tap("attn")
+    # a slot can be reloaded with the other form
+    seq_again = W.make_custom("again", W.SMALL, 3, MIXED, seed=32)
+    if flags & 1:
+        rng = np.random.default_rng(1)
+        for w in seq_again.weights:
+            w.update(W.draw_qk_norm(rng, W.SMALL))
+    B.upload_weights(ctx, seq_again.weights)
+    out2 = ctx.dit_step_forward_requests(B.bits_to_cuda_bf16(seq_again.packed_tokens()), seq_again.requests,
+                                         B.bits_to_cuda_bf16(seq_again.cond), 3)
+    torch.cuda.synchronize()
+    assert ctx.dit_last_launch_count() == 1 + 7 * 3
+    check(seq_again, out2, oracle_out(seq_again, rope=bool(flags & 2)))
+    ctx.close()
+
+
+def test_parallel_block_large_model(B):
+    wl = mixed_stack_workload(W.LARGE, "p", [(256, 256, 64), (128, 256, 0)], seed=33, qk_norm=True)
+    ctx, out = run_gpu(B, wl, 3)
+    check(wl, out, oracle_out(wl, rope=True))
+    ctx.close()
