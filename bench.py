@@ -114,7 +114,7 @@ def oracle_sample(wl: W.Workload):
     w0 = {k: W.bf16_to_f64(v) for k, v in wl.weights[0].items()}
 
     def run():
-        return O.block_forward(x, c, w0, wl.dims.n_heads, wl.dims.ln_eps)
+        return O.any_block_forward(x, c, w0, wl.dims.n_heads, wl.dims.ln_eps)
     req = wl.requests[r]
     desc = (f"request {r} of {wl.name} alone ({req.height}x{req.width}: {req.n_image_tokens} image + "
             f"{req.n_text_tokens} text tokens) through 1 of {wl.n_blocks} blocks, time scaled by {wl.n_blocks}; fp64 NumPy")
@@ -179,6 +179,10 @@ def run_gpu(args):
         nb = args.depth
         wl.weights = [wl.weights[b % len(wl.weights)] for b in range(nb)]
         wl.n_blocks = nb
+    if args.form == "parallel":
+        par_rng = np.random.default_rng(args.seed + 3000)
+        drawn = [W.draw_parallel_block_weights(par_rng, wl.dims) for _ in range(min(nb, 4))]
+        wl.weights = [drawn[b % len(drawn)] for b in range(nb)]
     if args.variants & 1:
         qk_rng = np.random.default_rng(args.seed + 2000)
         wl.weights = [dict(w, **W.draw_qk_norm(qk_rng, wl.dims)) for w in wl.weights]
@@ -325,7 +329,8 @@ def run_gpu(args):
     peaks = measured_peaks()
     H, F, T = wl.dims.hidden, wl.dims.mlp_hidden, wl.total_tokens
     per_launch_flops = {"gemm_qkv": 2.0 * T * H * 3 * H, "gemm_proj": 2.0 * T * H * H, "gemm_fc1": 2.0 * T * H * F,
-                        "gemm_fc2": 2.0 * T * H * F, "attention": 4.0 * H * sum(l * l for l in lens)}
+                        "gemm_fc2": 2.0 * T * H * (F + (H if args.form == "parallel" else 0)),   # parallel form: one K = H + F output GEMM
+                        "attention": 4.0 * H * sum(l * l for l in lens)}
     per_launch_bytes = {"ln_modulate": T * H * (4 + 2), "modulation": nb * wl.dims.cond_dim * 6 * H * 2}
     kern = {}
     for name, rec in kernels.items():
@@ -367,7 +372,7 @@ def run_gpu(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
-            "config": {"workload": wl.name, "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2)}, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
+            "config": {"workload": wl.name, "block_form": args.form, "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2)}, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
                        "total_tokens": T, "image_tokens": wl.image_tokens, "hidden": H, "heads": wl.dims.n_heads,
                        "head_dim": wl.dims.head_dim, "mlp_hidden": F, "parallelism": f"replicas x{world}",
                        "l2": "weights and activations of a step exceed L2 (126 MB); no flush"},
@@ -397,6 +402,8 @@ def main():
     ap.add_argument("--depth", type=int, default=0, help="run this many blocks instead of the configuration's (weights reused cyclically)")
     ap.add_argument("--variants", type=int, default=0, choices=[0, 1, 2, 3],
                     help="block variant bits: 1 = RMS-norm of queries and keys, 2 = 2-D rotary term (not the headline configuration)")
+    ap.add_argument("--form", default="sequential", choices=["sequential", "parallel"],
+                    help="block form: the adaLN-Zero block of the headline, or the parallel attention+MLP form (same FLOPs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
