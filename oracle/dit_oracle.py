@@ -33,6 +33,9 @@ of equal size, adjacent channel pairs, base 10000; text tokens at (0, 0)).
 A second block form, `parallel_block_forward`: one modulation triple, attention
 and MLP both read the same modulated LayerNorm output, one output projection
 over their concatenation (the "single-stream" blocks of the FLUX family).
+A third, `dual_block_forward`: image and text tokens of a request each have
+their own block tensors and meet only in attention (the "double-stream" /
+MMDiT blocks of the FLUX and SD3 families).
 
 Every function works on fp64 arrays.  Nothing is tiled, fused or reordered
 beyond taking query rows in slabs to bound memory (each softmax row is still
@@ -254,28 +257,71 @@ def parallel_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads:
     return y
 
 
-def any_block_forward(x, cond, w: Weights, n_heads: int, eps: float, **kw) -> np.ndarray:
-    """Dispatch on the block's form: a parallel block is the one that holds "w_out"."""
+def dual_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_img: int, n_heads: int, eps: float,
+                       rows: np.ndarray | None = None, taps: dict | None = None,
+                       positions: np.ndarray | None = None) -> np.ndarray:
+    """The two-stream form of the block: the first n_img rows (image tokens) use the tensors of
+    `w`, the remaining rows (text tokens) use those of w["txt"]; each stream has its own
+    modulation, projections, MLP and (optionally) q/k norm scales.  Only attention mixes them: it
+    runs once over all rows of the request, queries, keys and values taken stream by stream.
+    """
+    L, H = x.shape
+    streams = [(slice(0, n_img), w), (slice(n_img, L), w["txt"])]
+    mods, qs, ks, vs, hs = [], [], [], [], []
+    for sl, ws in streams:
+        m = adaln_modulation(cond, ws["w_ada"], ws["b_ada"])
+        h = modulate(layer_norm(x[sl], eps), m[0], m[1])
+        qkv = h @ ws["w_qkv"] + ws["b_qkv"]
+        q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
+        if "q_norm" in ws:
+            q = rms_norm_heads(q, ws["q_norm"], n_heads, eps)
+            k = rms_norm_heads(k, ws["k_norm"], n_heads, eps)
+        mods.append(m); hs.append(h); qs.append(q); ks.append(k); vs.append(v)
+    q, k, v = np.concatenate(qs), np.concatenate(ks), np.concatenate(vs)
+    if positions is not None:
+        q, k = rope_2d(q, positions, n_heads), rope_2d(k, positions, n_heads)
+    a = attention(q, k, v, n_heads)                      # all rows: both streams need their own
+    y = np.empty_like(x)
+    u_all = []
+    for (sl, ws), m in zip(streams, mods):
+        x_mid = x[sl] + m[2] * (a[sl] @ ws["w_o"] + ws["b_o"])
+        h2 = modulate(layer_norm(x_mid, eps), m[3], m[4])
+        u = gelu_tanh(h2 @ ws["w_fc1"] + ws["b_fc1"])
+        y[sl] = x_mid + m[5] * (u @ ws["w_fc2"] + ws["b_fc2"])
+        u_all.append(u)
+    if taps is not None:
+        taps.update(h1=np.concatenate(hs), qkv=np.concatenate([q, k, v], axis=1), a=a, u=np.concatenate(u_all))
+    return y if rows is None else y[rows]
+
+
+def any_block_forward(x, cond, w: Weights, n_heads: int, eps: float, n_img: int | None = None, **kw) -> np.ndarray:
+    """Dispatch on the block's form: a two-stream block holds "txt" (the text stream's tensors), a
+    parallel block holds "w_out".  n_img (image rows of the request) is needed by two-stream blocks."""
+    if "txt" in w:
+        return dual_block_forward(x, cond, w, n_img, n_heads, eps, **kw)
     return (parallel_block_forward if "w_out" in w else block_forward)(x, cond, w, n_heads, eps, **kw)
 
 
 def stack_forward_alone(x: np.ndarray, cond: np.ndarray, blocks: Sequence[Weights],
-                        n_heads: int, eps: float, positions: np.ndarray | None = None) -> np.ndarray:
+                        n_heads: int, eps: float, positions: np.ndarray | None = None,
+                        n_img: int | None = None) -> np.ndarray:
     """A stack of blocks on one request run by itself."""
     for w in blocks:
-        x = any_block_forward(x, cond, w, n_heads, eps, positions=positions)
+        x = any_block_forward(x, cond, w, n_heads, eps, n_img=n_img, positions=positions)
     return x
 
 
 def step_forward(packed: np.ndarray, token_lens: Sequence[int], cond: np.ndarray,
                  blocks: Sequence[Weights], n_heads: int, eps: float,
-                 positions: Sequence[np.ndarray] | None = None) -> np.ndarray:
+                 positions: Sequence[np.ndarray] | None = None,
+                 n_imgs: Sequence[int] | None = None) -> np.ndarray:
     """One denoising step over a packed batch: each request through the stack on its own."""
     out = np.empty_like(packed)
     p = 0
     for r, l in enumerate(token_lens):
         out[p:p + l] = stack_forward_alone(packed[p:p + l], cond[r], blocks, n_heads, eps,
-                                           None if positions is None else positions[r])
+                                           None if positions is None else positions[r],
+                                           None if n_imgs is None else n_imgs[r])
         p += l
     return out
 

@@ -149,7 +149,7 @@ def denoise_step(latents: Sequence[np.ndarray], texts: Sequence[np.ndarray], tim
         img = round_to_bf16(embed_latent(z, shell, hidden))
         tokens = img if txt.shape[0] == 0 else np.concatenate([img, txt], axis=0)
         pos = blocks.patch_positions(z.shape[1] * VAE_FACTOR, z.shape[2] * VAE_FACTOR, txt.shape[0]) if rope else None
-        x = blocks.stack_forward_alone(tokens, cond, block_ws, n_heads, eps, positions=pos)
+        x = blocks.stack_forward_alone(tokens, cond, block_ws, n_heads, eps, positions=pos, n_img=img.shape[0])
         v_tok = final_layer(x[:img.shape[0]], cond, shell, eps)
         v = unpatchify(v_tok, z.shape[1], z.shape[2])
         new_latents.append(euler_update(z, v, ds))

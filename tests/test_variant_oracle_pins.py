@@ -190,3 +190,58 @@ def test_parallel_block_zero_gate_rows_and_dispatch():
     seq = _block(rng, H, F, C)
     want = O.parallel_block_forward(O.block_forward(x, cond, seq, heads, 1e-6), cond, par, heads, 1e-6)
     assert np.array_equal(O.stack_forward_alone(x, cond, [seq, par], heads, 1e-6), want)
+
+
+# ----------------------------------------------------------------------------- the two-stream block form
+def test_dual_block_reduces_to_the_plain_block():
+    rng = np.random.default_rng(9)
+    H, F, C, heads, L, n_img = 64, 128, 8, 2, 7, 4
+    w_img, w_txt = _block(rng, H, F, C, d=32), _block(rng, H, F, C, d=32)
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    pos = np.array([[0, 0], [0, 1], [1, 0], [1, 1], [0, 0], [0, 0], [0, 0]])
+    # same tensors in both streams: the plain block
+    same = dict(w_img, txt=w_img)
+    assert np.allclose(O.dual_block_forward(x, cond, same, n_img, heads, 1e-6, positions=pos),
+                       O.block_forward(x, cond, w_img, heads, 1e-6, positions=pos), atol=1e-13)
+    dual = dict(w_img, txt=w_txt)
+    # no text rows: the image stream's plain block; no image rows: the text stream's
+    assert np.allclose(O.dual_block_forward(x, cond, dual, L, heads, 1e-6), O.block_forward(x, cond, w_img, heads, 1e-6), atol=1e-13)
+    assert np.allclose(O.dual_block_forward(x, cond, dual, 0, heads, 1e-6), O.block_forward(x, cond, w_txt, heads, 1e-6), atol=1e-13)
+    # different tensors: a different result, and the boundary matters
+    y = O.dual_block_forward(x, cond, dual, n_img, heads, 1e-6, positions=pos)
+    assert not np.allclose(y, O.block_forward(x, cond, w_img, heads, 1e-6, positions=pos), atol=1e-3)
+    assert not np.allclose(y, O.dual_block_forward(x, cond, dual, n_img + 1, heads, 1e-6, positions=pos), atol=1e-3)
+
+
+def test_dual_block_streams_meet_only_in_attention():
+    rng = np.random.default_rng(10)
+    H, F, C, heads, L, n_img = 64, 128, 8, 2, 6, 4
+    w_img, w_txt = _block(rng, H, F, C), _block(rng, H, F, C)
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    dual = dict(w_img, txt=w_txt)
+    y = O.dual_block_forward(x, cond, dual, n_img, heads, 1e-6)
+    # zero gates in the text stream: text rows pass through, image rows still change (and still see
+    # the text keys and values, which do not depend on the gates)
+    wz = dict(w_txt, w_ada=w_txt["w_ada"].copy(), b_ada=w_txt["b_ada"].copy())
+    for g in (2, 5):
+        wz["w_ada"][:, g * H:(g + 1) * H] = 0.0
+        wz["b_ada"][g * H:(g + 1) * H] = 0.0
+    yz = O.dual_block_forward(x, cond, dict(w_img, txt=wz), n_img, heads, 1e-6)
+    assert np.array_equal(yz[n_img:], x[n_img:])
+    assert np.allclose(yz[:n_img], y[:n_img], atol=1e-13)
+    # text values projected to zero: image rows attend to nothing of the text but its softmax mass;
+    # hand check on the attention tap: rows of `a` are convex combinations of the value rows
+    taps = {}
+    O.dual_block_forward(x, cond, dual, n_img, heads, 1e-6, taps=taps)
+    v = taps["qkv"][:, 2 * H:]
+    a = taps["a"]
+    for j in range(heads):
+        cols = slice(j * 32, (j + 1) * 32)
+        assert (a[:, cols].max(0) <= v[:, cols].max(0) + 1e-12).all() and (a[:, cols].min(0) >= v[:, cols].min(0) - 1e-12).all()
+    # the text stream's MLP does not touch image rows: change only w_fc2 of the text stream
+    w2 = dict(w_txt, w_fc2=w_txt["w_fc2"] * 3.0)
+    y2 = O.dual_block_forward(x, cond, dict(w_img, txt=w2), n_img, heads, 1e-6)
+    assert np.array_equal(y2[:n_img], y[:n_img]) and not np.allclose(y2[n_img:], y[n_img:], atol=1e-3)
+    # row subset and stack dispatch
+    assert np.array_equal(O.dual_block_forward(x, cond, dual, n_img, heads, 1e-6, rows=np.array([5, 0])), y[[5, 0]])
+    assert np.array_equal(O.stack_forward_alone(x, cond, [dual], heads, 1e-6, n_img=n_img), y)
