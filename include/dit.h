@@ -139,6 +139,19 @@ typedef struct {
 dit_status dit_load_parallel_block_weights(dit_ctx *ctx, int32_t block_idx, const dit_parallel_block_weights *w,
                                            void *stream);
 
+/* The two-stream form of the block (the double-stream / MMDiT blocks of the FLUX and SD3 families):
+ * image tokens and text tokens of a request each have their own ten tensors (modulation, projections,
+ * MLP, and q/k norm scales) and meet only in attention, which runs once over all tokens of the
+ * request.  Such a block occupies TWO consecutive slots, block_idx (image stream) and block_idx + 1
+ * (text stream); n_blocks of the step calls counts slots.  Loading either slot on its own later
+ * dissolves the pair.  It needs the requests' geometry to tell image rows from text rows:
+ * dit_step_forward_requests or dit_denoise_step.  Inside, every GEMM of the block visits the 256-row
+ * tiles stream by stream with that stream's weights; a tile that holds rows of both streams is
+ * computed once per stream and each pass stores its own rows (with the paper's token counts,
+ * multiples of 256 image tokens and 512 text tokens, no tile is mixed). */
+dit_status dit_load_dual_block_weights(dit_ctx *ctx, int32_t block_idx, const dit_block_weights *image_stream,
+                                       const dit_block_weights *text_stream, void *stream);
+
 /* Packer, host only, integer only (Section 6.1 token rule; requests keep their input order; inside
  * a request image tokens come first, then text tokens).  All arrays are HOST memory owned by the
  * caller: token_lens [n], cu_seqlens [n+1], row_req / row_local [sum of lens] (either may be NULL).

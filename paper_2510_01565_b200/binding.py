@@ -23,7 +23,7 @@ STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPAC
 KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
-EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights",
+EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights", "dit_load_dual_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
            "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
@@ -96,6 +96,8 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_destroy.argtypes = [vp]
     lib.dit_load_block_weights.restype = C.c_int
     lib.dit_load_block_weights.argtypes = [vp, i32, C.POINTER(DitBlockWeights), vp]
+    lib.dit_load_dual_block_weights.restype = C.c_int
+    lib.dit_load_dual_block_weights.argtypes = [vp, i32, C.POINTER(DitBlockWeights), C.POINTER(DitBlockWeights), vp]
     lib.dit_load_parallel_block_weights.restype = C.c_int
     lib.dit_load_parallel_block_weights.argtypes = [vp, i32, C.POINTER(DitParallelBlockWeights), vp]
     lib.dit_pack_requests.restype = C.c_int
@@ -272,19 +274,27 @@ class DitContext:
             pass
 
     # ------------------------------------------------------------------ C-ABI calls
-    def dit_load_block_weights(self, block_idx: int, weights: Dict[str, "object"], stream=None):
-        """weights: name -> CUDA bf16 tensor, [in, out] row-major; biases may be None."""
+    def _block_struct(self, weights: Dict[str, "object"]) -> DitBlockWeights:
         w = DitBlockWeights()
-        keep = []
         for name, _ in DitBlockWeights._fields_:
             t = weights.get(name)
             if t is None:
                 setattr(w, name, None)
                 continue
             assert t.is_cuda and t.dtype == self.torch.bfloat16 and t.is_contiguous(), name
-            keep.append(t)
             setattr(w, name, t.data_ptr())
+        return w
+
+    def dit_load_block_weights(self, block_idx: int, weights: Dict[str, "object"], stream=None):
+        """weights: name -> CUDA bf16 tensor, [in, out] row-major; biases may be None."""
+        w = self._block_struct(weights)
         self._check(self.lib.dit_load_block_weights(self.handle, block_idx, C.byref(w), self._stream(stream)))
+
+    def dit_load_dual_block_weights(self, block_idx: int, image_stream: Dict[str, "object"],
+                                    text_stream: Dict[str, "object"], stream=None):
+        """Two-stream block in slots block_idx (image tokens) and block_idx + 1 (text tokens)."""
+        wi, wt = self._block_struct(image_stream), self._block_struct(text_stream)
+        self._check(self.lib.dit_load_dual_block_weights(self.handle, block_idx, C.byref(wi), C.byref(wt), self._stream(stream)))
 
     def dit_load_parallel_block_weights(self, block_idx: int, weights: Dict[str, "object"], stream=None):
         """Parallel-form block: name -> CUDA bf16 tensor ([in, out] row-major); biases and norms may be None."""
@@ -497,17 +507,30 @@ def context_for(dims, max_blocks: int, max_total_tokens: int, max_requests: int 
                       max_blocks, max_total_tokens, max_requests, dims.ln_eps, flags)
 
 
-def upload_weights(ctx: DitContext, blocks) -> None:
-    """blocks: list of dicts name -> numpy uint16 (bf16 bits).  Copies to the GPU and loads them."""
+def upload_weights(ctx: DitContext, blocks) -> int:
+    """blocks: list of dicts name -> numpy uint16 (bf16 bits).  Copies to the GPU and loads them.
+
+    A dict with "w_out" is a parallel-form block; a dict with "txt" (the text stream's dict) is a
+    two-stream block and takes two slots.  Returns the number of slots used (n_blocks of a step).
+    """
     import torch
-    for b, w in enumerate(blocks):
-        dev = {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in w.items()}
-        if "w_out" in w:          # the parallel form of the block
-            ctx.dit_load_parallel_block_weights(b, dev)
+    to_dev = lambda w: {k: torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16) for k, v in w.items() if k != "txt"}
+    slot = 0
+    for w in blocks:
+        dev = to_dev(w)
+        if "txt" in w:
+            txt = to_dev(w["txt"])
+            ctx.dit_load_dual_block_weights(slot, dev, txt)
+            slot += 2
+        elif "w_out" in w:
+            ctx.dit_load_parallel_block_weights(slot, dev)
+            slot += 1
         else:
-            ctx.dit_load_block_weights(b, dev)
+            ctx.dit_load_block_weights(slot, dev)
+            slot += 1
         torch.cuda.synchronize()
         del dev
+    return slot
 
 
 def upload_shell_weights(ctx: DitContext, shell) -> None:

@@ -41,4 +41,9 @@ __device__ __forceinline__ int find_request(const SeqInfo& s, int row) {
   return lo;
 }
 
+// 0 for an image token, 1 for a text token (two-stream blocks choose their tensors by this).
+__device__ __forceinline__ int row_kind(const SeqInfo& s, const RowGeom& g, int req, int row) {
+  return (row - s.cu[req]) >= (g.img_cu[req + 1] - g.img_cu[req]) ? 1 : 0;
+}
+
 }  // namespace dit

@@ -38,6 +38,7 @@ struct Layout {
   size_t sh_w_in, sh_b_in, sh_w_t1, sh_b_t1, sh_w_t2, sh_b_t2, sh_w_fa, sh_b_fa, sh_w_out, sh_b_out;
   size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok;
   size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
+  size_t items;        // two-stream launches: [0] item count, then per-tile flags, then the items
   size_t bytes;
 };
 constexpr int kWoutRows = 256;   // W_out^T is stored zero-padded to one full weight tile of the GEMM
@@ -103,6 +104,7 @@ Layout make_layout(const dit_config& c) {
   L.sh_modfin = take(R * 2 * H * 4);
   L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
   L.rope_theta = take(64 * 4);
+  L.items = take((16 + 3 * (T / (2 * 128) + 2)) * 4);
   L.bytes = o;
   return L;
 }
@@ -110,6 +112,8 @@ Layout make_layout(const dit_config& c) {
 struct BlockState {
   bool loaded = false;
   bool parallel = false;                   // parallel form: tm_o is unused, tm_fc2 maps W_out^T [H, H + F]
+  bool dual = false;                       // image stream of a two-stream block; the text stream is the next slot
+  bool dual_second = false;                // text stream of a two-stream block (run together with the slot before)
   CUtensorMap tm_qkv, tm_o, tm_fc1, tm_fc2;
 };
 
@@ -180,17 +184,17 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
 
 const RowGeom kNoGeom{};
 
-template <int EPI, int HD = 0>
+template <int EPI, int HD = 0, bool DUAL = false>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
-                        const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom) {
+                        const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom, const CUtensorMap* tmB2 = nullptr) {
   // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
   GemmParams q = p;
   const long long band_bytes = 2ll * gemm_cfg::BM * p.K * 2;
   q.band = static_cast<int>(std::max(1ll, std::min<long long>((36ll << 20) / band_bytes, (p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM))));
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
-  const int grid = 2 * std::min(tiles, ctx->gemm_pairs);
-  gemm_tcgen05_kernel<EPI, HD><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, q, seq, geo);
+  const int grid = 2 * std::min(tiles, ctx->gemm_pairs);   // a two-stream launch may have more items than row tiles: the loop covers them
+  gemm_tcgen05_kernel<EPI, HD, DUAL><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
   return cudaGetLastError();
 }
 
@@ -205,11 +209,12 @@ cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, cons
 // LayerNorm + modulate launch: picks the register-resident row width (float4 per lane) for H.
 template <bool kFromBf16>
 cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
-                      long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st) {
+                      long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st,
+                      long long kind_stride = 0, const RowGeom& geo = kNoGeom) {
   const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
-  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
-  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
-  else ln_modulate_kernel<kFromBf16, 32><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq);
+  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
+  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
+  else ln_modulate_kernel<kFromBf16, 32><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
   return cudaGetLastError();
 }
 
@@ -287,14 +292,47 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }));
   }
 
+  // two-stream blocks: validate the pairing and list the row tiles of each stream once per step
+  bool any_dual = false;
+  for (int b = 0; b < n_blocks; ++b) {
+    if (!ctx->blocks[b].dual) continue;
+    any_dual = true;
+    if (b + 1 >= n_blocks || !ctx->blocks[b + 1].dual_second)
+      return fail(ctx, DIT_ERR_INVALID_ARG, "n_blocks ends between the two slots of a two-stream block");
+  }
+  if (ctx->blocks[0].dual_second) return fail(ctx, DIT_ERR_INVALID_ARG, "slot 0 holds the second half of a two-stream block");
+  if (any_dual && !geo)
+    return fail(ctx, DIT_ERR_INVALID_ARG, "two-stream blocks need the requests' geometry: use dit_step_forward_requests");
+  const RowGeom& rg = geo ? *geo : kNoGeom;
+  int* item_count = ctx->at<int>(ctx->lay.items);
+  int* item_flags = item_count + 16;
+  int* items = item_flags + (c.max_total_tokens / (2 * gemm_cfg::BM) + 2);
+  if (any_dual) {
+    build_row_items_kernel<<<1, 256, 0, st>>>(seq, rg, 2 * gemm_cfg::BM, item_flags, items, item_count);
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+    ++launches;
+  }
+
   for (int b = 0; b < n_blocks; ++b) {
     const BlockState& bs = ctx->blocks[b];
+    if (bs.dual_second) continue;                      // ran together with the slot before
+    const bool dual = bs.dual;
+    const BlockState& bt = ctx->blocks[dual ? b + 1 : b];     // text stream's slot of a two-stream block
     const uint8_t* wb = ctx->block_base(b);
+    const uint8_t* wt = ctx->block_base(dual ? b + 1 : b);
+    const long long ks = dual ? 6ll * H : 0;           // text stream's modulation vectors follow the image stream's
+    const bool last = (dual ? b + 1 : b) == n_blocks - 1;
     const float* modb = mod + static_cast<size_t>(b) * 6 * H;   // request 0; request r at + r * req_stride
+    auto two_stream = [&](GemmParams& gp, size_t bias_off) {
+      if (!dual) return;
+      gp.items = items; gp.num_items = item_count;
+      gp.bias2 = reinterpret_cast<const float*>(wt + bias_off);
+      gp.gate_kind_stride = ks;
+    };
     // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st)
-                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st);
+      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg)
+                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
     }));
     // QKV projection
     GemmParams g{};
@@ -302,22 +340,30 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.M = T; g.N = 3 * H; g.K = H;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_qkv);
     g.out16 = qkv;
+    two_stream(g, ctx->lay.blk.b_qkv);
     if (qk_variant) {
       g.hidden = H; g.eps = c.ln_eps;
       if (c.flags & DIT_FLAG_QK_RMSNORM) {
         g.q_norm = reinterpret_cast<const float*>(wb + ctx->lay.blk.q_norm);
         g.k_norm = reinterpret_cast<const float*>(wb + ctx->lay.blk.k_norm);
+        g.q_norm2 = reinterpret_cast<const float*>(wt + ctx->lay.blk.q_norm);
+        g.k_norm2 = reinterpret_cast<const float*>(wt + ctx->lay.blk.k_norm);
       }
       if (c.flags & DIT_FLAG_ROPE_2D) g.rope_theta = ctx->at<float>(ctx->lay.rope_theta);
-      const RowGeom& rg = geo ? *geo : kNoGeom;
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+        if (dual)
+          return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
+                                   : launch_gemm<kEpiQkvF16, 64, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv);
         return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg)
                                  : launch_gemm<kEpiQkvF16, 64>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg);
       }));
     } else {
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] { return launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st); }));
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+        return dual ? launch_gemm<kEpiBiasF16, 0, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
+                    : launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st);
+      }));
     }
-    // attention
+    // attention (one pass over all tokens of a request, whatever their stream)
     AttnParams ap{};
     ap.out = bs.parallel ? cat : a; ap.ld_out = bs.parallel ? H + F : H;
     ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
@@ -341,7 +387,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       g.status = status;
       g.M = T; g.N = H; g.K = H + F;
       g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
-      g.resid = stream; g.out32 = (b == n_blocks - 1) ? out : stream;
+      g.resid = stream; g.out32 = last ? out : stream;
       g.gate = modb + 2 * H; g.gate_stride = req_stride;
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
       continue;
@@ -353,10 +399,14 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_o);
     g.resid = stream; g.out32 = stream;
     g.gate = modb + 2 * H; g.gate_stride = req_stride;
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st); }));
+    two_stream(g, ctx->lay.blk.b_o);
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] {
+      return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_a, bs.tm_o, g, seq, st, rg, &bt.tm_o)
+                  : launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st);
+    }));
     // LN2 + modulate
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      return launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st);
+      return launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
     }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};
@@ -364,20 +414,37 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.M = T; g.N = F; g.K = H;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
     g.out16 = u;
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st); }));
+    two_stream(g, ctx->lay.blk.b_fc1);
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
+      return dual ? launch_gemm<kEpiBiasGeluF16, 0, true>(ctx, tm_h, bs.tm_fc1, g, seq, st, rg, &bt.tm_fc1)
+                  : launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st);
+    }));
     // MLP down-projection + gate + residual (last block writes the caller's output)
     g = GemmParams{};
     g.status = status;
     g.M = T; g.N = H; g.K = F;
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
-    g.resid = stream; g.out32 = (b == n_blocks - 1) ? out : stream;
+    g.resid = stream; g.out32 = last ? out : stream;
     g.gate = modb + 5 * H; g.gate_stride = req_stride;
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st); }));
+    two_stream(g, ctx->lay.blk.b_fc2);
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] {
+      return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_u, bs.tm_fc2, g, seq, st, rg, &bt.tm_fc2)
+                  : launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st);
+    }));
   }
   ctx->last_launches = launches;
   ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
   ctx->last_parallel = ctx->blocks[n_blocks - 1].parallel;
   return DIT_OK;
+}
+
+// Loading one slot on its own dissolves a two-stream pair it was part of: the other half must be
+// loaded again before it can run.
+void unpair_slot(dit_ctx* ctx, int b) {
+  BlockState& bs = ctx->blocks[b];
+  if (bs.dual && b + 1 < ctx->cfg.max_blocks) { ctx->blocks[b + 1].dual_second = false; ctx->blocks[b + 1].loaded = false; }
+  if (bs.dual_second && b > 0) { ctx->blocks[b - 1].dual = false; ctx->blocks[b - 1].loaded = false; }
+  bs.dual = bs.dual_second = false;
 }
 
 dit_status check_step_args(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
@@ -457,6 +524,11 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF32>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16, 0, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16, 0, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32, 0, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>), mod_smem_bytes(kMaxCondDim));  // same for every context
@@ -505,6 +577,7 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   uint8_t* base = ctx->block_base(b);
   const BlockLayout& L = ctx->lay.blk;
   BlockState& bs = ctx->blocks[b];
+  unpair_slot(ctx, b);
   bs.loaded = false;
   bs.parallel = false;
 
@@ -539,6 +612,20 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   return DIT_OK;
 }
 
+dit_status dit_load_dual_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weights* image_stream,
+                                       const dit_block_weights* text_stream, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (b < 0 || b + 1 >= ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "a two-stream block needs slots b and b + 1 inside [0, max_blocks)");
+  dit_status s = dit_load_block_weights(ctx, b, image_stream, stream);
+  if (s != DIT_OK) return s;
+  s = dit_load_block_weights(ctx, b + 1, text_stream, stream);
+  if (s != DIT_OK) return s;
+  ctx->blocks[b].dual = true;
+  ctx->blocks[b + 1].dual_second = true;
+  return DIT_OK;
+}
+
 dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_parallel_block_weights* w, void* stream) {
   if (!ctx) return DIT_ERR_INVALID_ARG;
   ctx->err[0] = 0;
@@ -550,6 +637,7 @@ dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_pa
   uint8_t* base = ctx->block_base(b);
   const BlockLayout& L = ctx->lay.blk;
   BlockState& bs = ctx->blocks[b];
+  unpair_slot(ctx, b);
   bs.loaded = false;
   bs.parallel = true;
 

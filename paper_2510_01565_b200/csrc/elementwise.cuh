@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 // statistics, fixed shuffle order.  Small CTAs (4 rows) and a register budget that lets several CTAs
 // share an SM keep enough loads in flight to cover HBM latency.
 // kFromBf16 = true reads the packed bf16 tokens (first block) and also writes the fp32 residual stream.
+// kind_stride != 0: two-stream block, the modulation vectors are chosen per row by image/text.
 // ------------------------------------------------------------------------------------------------
 constexpr int kLnWarps = 4;
 
@@ -143,7 +144,8 @@ template <bool kFromBf16, int kLnMaxVec>
 __global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVec <= 24 ? 4 : 3)))
 ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
                    const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
-                   int T, int H, float eps, const __grid_constant__ SeqInfo seq) {
+                   int T, int H, float eps, const __grid_constant__ SeqInfo seq,
+                   long long kind_stride, const __grid_constant__ RowGeom geo) {
   const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= T) return;
@@ -180,8 +182,10 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
   for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
   const float rstd = rsqrtf(sq / static_cast<float>(H) + eps);
   const int req = find_request(seq, row);
-  const float4* sh = reinterpret_cast<const float4*>(shift0 + req * req_stride);
-  const float4* sc = reinterpret_cast<const float4*>(scale0 + req * req_stride);
+  // two-stream blocks: text tokens take the text stream's vectors, kind_stride floats further on
+  const long long voff = req * req_stride + (kind_stride ? row_kind(seq, geo, req, row) * kind_stride : 0);
+  const float4* sh = reinterpret_cast<const float4*>(shift0 + voff);
+  const float4* sc = reinterpret_cast<const float4*>(scale0 + voff);
   uint2* dst = reinterpret_cast<uint2*>(h + static_cast<size_t>(row) * H);
 #pragma unroll
   for (int i = 0; i < kLnMaxVec; ++i) {
@@ -195,6 +199,37 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
       const __half2 lo = __floats2half2_rn(a, b), hi = __floats2half2_rn(c, d);
       dst[idx] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row-tile items of a two-stream GEMM launch: for every tile of `tile_rows` packed rows, one item per
+// stream (image = 0, text = 1) that has at least one row in the tile, in row order.  One small CTA;
+// the compaction is serial (a batch has at most a few thousand row tiles).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+build_row_items_kernel(const __grid_constant__ SeqInfo seq, const __grid_constant__ RowGeom geo, int tile_rows,
+                       int* __restrict__ flags, int* __restrict__ items, int* __restrict__ num_items) {
+  const int num_m = (seq.total + tile_rows - 1) / tile_rows;
+  for (int mb = threadIdx.x; mb < num_m; mb += blockDim.x) {
+    const int lo = mb * tile_rows, hi = min(seq.total, lo + tile_rows);
+    int f = 0;
+    for (int r = find_request(seq, lo); r < seq.n && seq.cu[r] < hi; ++r) {
+      const int img_end = seq.cu[r] + (geo.img_cu[r + 1] - geo.img_cu[r]);
+      if (max(lo, seq.cu[r]) < min(hi, img_end)) f |= 1;
+      if (max(lo, img_end) < min(hi, seq.cu[r + 1])) f |= 2;
+    }
+    flags[mb] = f;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int mb = 0; mb < num_m; ++mb) {
+      const int f = flags[mb];
+      if (f & 1) items[n++] = mb;
+      if (f & 2) items[n++] = mb | (1 << 24);
+    }
+    *num_items = n;
   }
 }
 

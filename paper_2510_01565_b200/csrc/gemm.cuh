@@ -46,6 +46,14 @@ struct GemmParams {
   const float* rope_theta;  // [(HD - HD/8) / 4] pair frequencies of one axis group, NULL = no rotary term
   int hidden;               // H: columns [0,H) are Q, [H,2H) K, [2H,3H) V
   float eps;
+  // two-stream launches (DUAL) only: row-tile items, and the text stream's epilogue tensors
+  const int* items;         // item i = row tile (low 24 bits) | stream << 24; a tile holding rows of both
+                            // streams appears twice and each pass stores only its own stream's rows
+  const int* num_items;
+  const float* bias2;       // text stream's bias
+  const float* q_norm2;
+  const float* k_norm2;
+  long long gate_kind_stride;   // text stream's gate vector = gate + gate_kind_stride
 };
 
 namespace gemm_cfg {
@@ -78,10 +86,14 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int ban
   mb = b * band + (r - nb * rows);
 }
 
-template <int EPI, int HD = 0>
+// DUAL: two-stream launch.  The weight operand comes from tmB for image-token rows and from tmB2 for
+// text-token rows; the row tiles to visit are listed in p.items (built on the device from the batch's
+// geometry), everything else is unchanged.
+template <int EPI, int HD = 0, bool DUAL = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmParams p, const __grid_constant__ SeqInfo seq, const __grid_constant__ RowGeom geo) {
+                    const __grid_constant__ CUtensorMap tmB2, const GemmParams p,
+                    const __grid_constant__ SeqInfo seq, const __grid_constant__ RowGeom geo) {
   using namespace gemm_cfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -101,8 +113,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                    // 0 = leader of the pair
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int num_m = (p.M + 2 * BM - 1) / (2 * BM), num_n = (p.N + BN - 1) / BN;
+  const int num_m = DUAL ? *p.num_items : (p.M + 2 * BM - 1) / (2 * BM);   // row tiles (DUAL: row-tile items)
+  const int num_n = (p.N + BN - 1) / BN;
   const int num_tiles = num_m * num_n;                        // 256 x 256 tiles
+  // row tile and stream of item ib
+  auto item_of = [&](int ib, int& mb, int& kind) {
+    if (DUAL) { const int it = __ldg(p.items + ib); mb = it & 0xFFFFFF; kind = it >> 24; }
+    else { mb = ib; kind = 0; }
+  };
   const int num_k = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -111,7 +129,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 0 && lane == 0) { prefetch_tmap(&tmA); prefetch_tmap(&tmB); }
+  if (warp == 0 && lane == 0) { prefetch_tmap(&tmA); prefetch_tmap(&tmB); if (DUAL) prefetch_tmap(&tmB2); }
   if (warp == 1) { tmem_alloc_pair(smem_u32(tmem_slot), 512); tmem_relinquish_pair(); }
   tc_fence_before();
   __syncthreads();
@@ -124,8 +142,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       for (int t = pair; t < num_tiles; t += num_pairs) {
-        int mb, nb;
-        tile_coords(t, num_m, num_n, p.band, mb, nb);
+        int ib, mb, nb, kind;
+        tile_coords(t, num_m, num_n, p.band, ib, nb);
+        item_of(ib, mb, kind);
+        const CUtensorMap* tb = (DUAL && kind) ? &tmB2 : &tmB;
         const int m0 = mb * (2 * BM) + rank * BM;             // this CTA's rows of A
         const int n0 = nb * BN + rank * (BN / 2);             // this CTA's half of the weight tile
         for (int kb = 0; kb < num_k; ++kb) {
@@ -134,7 +154,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE_BYTES);   // both CTAs' bytes
           const uint32_t sa = base + stage * STAGE_BYTES;
           tma_load_2d_pair(sa, &tmA, kb * BK, m0, full_leader);
-          tma_load_2d_pair(sa + A_BYTES, &tmB, kb * BK, n0, full_leader);
+          tma_load_2d_pair(sa + A_BYTES, tb, kb * BK, n0, full_leader);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -171,14 +191,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
     for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
       const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
-      int mb, nb;
-      tile_coords(t, num_m, num_n, p.band, mb, nb);
+      int ib, mb, nb, kind;
+      tile_coords(t, num_m, num_n, p.band, ib, nb);
+      item_of(ib, mb, kind);
       const int m0 = mb * (2 * BM) + rank * BM, n0 = nb * BN;
       const int row = m0 + quarter * 32 + lane;
-      const bool row_ok = row < p.M;
       // gated-residual epilogue: request of this lane's row, and whether the warp's rows share it
       int my_req = -1;
-      if (EPI == kEpiGateResidF32 && row_ok) my_req = find_request(seq, row);
+      if ((EPI == kEpiGateResidF32 || DUAL) && row < p.M) my_req = find_request(seq, row);
+      // two-stream launch: this pass stores only the rows of its own stream
+      int my_kind = -1;
+      if (DUAL && row < p.M) my_kind = row_kind(seq, geo, my_req, row);
+      const bool row_ok = row < p.M && (!DUAL || my_kind == kind);
+      const float* bias = (DUAL && kind) ? p.bias2 : p.bias;
+      const float* gate = p.gate + ((DUAL && kind) ? p.gate_kind_stride : 0);
       const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
       const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
       // Residual rows of this tile do not depend on the accumulator: the first two 32-column chunks
@@ -220,12 +246,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             tmem_ld32(t_row + hc * HD + q * 32, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[q * 32 + i] = __uint_as_float(r[i]) + __ldg(p.bias + colh + q * 32 + i);
+            for (int i = 0; i < 32; ++i) v[q * 32 + i] = __uint_as_float(r[i]) + __ldg(bias + colh + q * 32 + i);
           }
           if (row_ok) {
-            const int kind = colh / p.hidden;  // 0 = Q, 1 = K, 2 = V
-            if (kind < 2) {
-              const float* g = kind == 0 ? p.q_norm : p.k_norm;
+            const int part = colh / p.hidden;  // 0 = Q, 1 = K, 2 = V
+            if (part < 2) {
+              const float* g = (DUAL && kind) ? (part == 0 ? p.q_norm2 : p.k_norm2) : (part == 0 ? p.q_norm : p.k_norm);
               if (g) {
                 float ss = 0.f;
 #pragma unroll
@@ -284,9 +310,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           __syncwarp();
           const int col = col0 + cg;                        // N is a multiple of 64: the whole chunk is inside
           {
-            const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + col));
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(p.gate + req0 * p.gate_stride + col));
+            if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(gate + req0 * p.gate_stride + col));
             float4 x[8];
             if (EPI == kEpiGateResidF32) {
 #pragma unroll
@@ -298,8 +324,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               const int rr = it * 4 + (lane >> 3);
               const int grow = m0 + quarter * 32 + rr;
               const int rq = __shfl_sync(0xffffffffu, my_req, rr);
-              if (grow < p.M) {
-                if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(p.gate + rq * p.gate_stride + col));
+              const int rk = DUAL ? __shfl_sync(0xffffffffu, my_kind, rr) : 0;
+              if (grow < p.M && (!DUAL || rk == kind)) {
+                if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(gate + rq * p.gate_stride + col));
                 const float* a = st + rr * 33 + cg;
                 float4 o;
                 if (EPI == kEpiGateResidF32) {
@@ -325,8 +352,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
                 const int i = 8 * v + 2 * h;
-                float a = __uint_as_float(r[i]) + __ldg(p.bias + col0 + i);
-                float b = __uint_as_float(r[i + 1]) + __ldg(p.bias + col0 + i + 1);
+                float a = __uint_as_float(r[i]) + __ldg(bias + col0 + i);
+                float b = __uint_as_float(r[i + 1]) + __ldg(bias + col0 + i + 1);
                 if (EPI == kEpiBiasGeluF16) { a = gelu_tanh_f32(a); b = gelu_tanh_f32(b); }
                 const __half2 hh = __floats2half2_rn(a, b);
                 w[h] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -337,7 +364,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               if (col0 + i < p.N) {
-                float a = __uint_as_float(r[i]) + p.bias[col0 + i];
+                float a = __uint_as_float(r[i]) + bias[col0 + i];
                 if (EPI == kEpiBiasGeluF16) a = gelu_tanh_f32(a);
                 dst[i] = __float2half_rn(a);
               }

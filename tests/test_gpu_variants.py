@@ -220,3 +220,88 @@ def test_parallel_block_large_model(B):
     ctx, out = run_gpu(B, wl, 3)
     check(wl, out, oracle_out(wl, rope=True))
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- the two-stream block form
+def dual_stack_workload(dims, kinds, reqs, seed, qk_norm):
+    """kinds: 's' sequential, 'p' parallel, 'd' two-stream, per block."""
+    wl = W.make_custom("stack", dims, len(kinds), reqs, seed=seed)
+    rng = np.random.default_rng(seed + 900)
+    for b, kind in enumerate(kinds):
+        if kind == "p":
+            wl.weights[b] = W.draw_parallel_block_weights(rng, dims)
+        if kind == "d":
+            wl.weights[b]["txt"] = W.draw_block_weights(rng, dims)
+        if qk_norm:
+            wl.weights[b].update(W.draw_qk_norm(rng, dims))
+            if kind == "d":
+                wl.weights[b]["txt"].update(W.draw_qk_norm(rng, dims))
+    return wl
+
+
+def f64_blocks(wl):
+    out = []
+    for w in wl.weights:
+        d = {k: W.bf16_to_f64(v) for k, v in w.items() if k != "txt"}
+        if "txt" in w:
+            d["txt"] = f64w(w["txt"])
+        out.append(d)
+    return out
+
+
+def run_stack(B, wl, flags):
+    import torch
+    slots = sum(2 if "txt" in w else 1 for w in wl.weights)
+    ctx = B.context_for(wl.dims, slots, wl.total_tokens, len(wl.requests), flags=flags)
+    assert B.upload_weights(ctx, wl.weights) == slots
+    tok, cond = B.bits_to_cuda_bf16(wl.packed_tokens()), B.bits_to_cuda_bf16(wl.cond)
+    out = ctx.dit_step_forward_requests(tok, wl.requests, cond, slots)
+    torch.cuda.synchronize()
+    ctx.dit_ctx_poll_status()
+    return ctx, out, slots, tok, cond
+
+
+def stack_oracle(wl, rope):
+    pos = [O.patch_positions(q.height, q.width, q.n_text_tokens) for q in wl.requests] if rope else None
+    return O.step_forward(W.bf16_to_f64(wl.packed_tokens()), wl.token_lens, W.bf16_to_f64(wl.cond), f64_blocks(wl),
+                          wl.dims.n_heads, wl.dims.ln_eps, positions=pos, n_imgs=[q.n_image_tokens for q in wl.requests])
+
+
+@pytest.mark.parametrize("flags", [0, 3])
+def test_two_stream_blocks_ragged_batch(B, flags):
+    # every 256-row tile of this batch holds rows of both streams and of several requests
+    import torch
+    wl = dual_stack_workload(W.SMALL, "dsdp", MIXED + [(64, 64, 40)], seed=41, qk_norm=bool(flags & 1))
+    ctx, out, slots, tok, cond = run_stack(B, wl, flags)
+    assert slots == 6 and ctx.dit_last_launch_count() == 1 + 1 + 7 + 7 + 7 + 5
+    check(wl, out, stack_oracle(wl, rope=bool(flags & 2)))
+    cu = np.concatenate([[0], np.cumsum(wl.token_lens)])
+    for r in (0, 3, 4):
+        a, b = int(cu[r]), int(cu[r + 1])
+        alone = ctx.dit_step_forward_requests(tok[a:b].contiguous(), [wl.requests[r]], cond[r:r + 1].contiguous(), slots)
+        torch.cuda.synchronize()
+        assert torch.equal(alone, out[a:b]), f"request {r}: packed and alone outputs differ"
+    # the pair cannot be cut, and bare lengths do not tell image rows from text rows
+    with pytest.raises(B.DitError) as e:
+        ctx.dit_step_forward_requests(tok, wl.requests, cond, 1)
+    assert e.value.status == 1
+    with pytest.raises(B.DitError) as e:
+        ctx.dit_step_forward(tok, wl.token_lens, cond, slots)
+    assert e.value.status == 1
+    ctx.close()
+
+
+def test_two_stream_block_pure_and_mixed_tiles(B):
+    # 256 image + 256 text tokens per request: every tile belongs to one stream; a third request
+    # (64 + 100 tokens) adds tiles that mix streams and requests
+    wl = dual_stack_workload(W.SMALL, "dd", [(256, 256, 256), (256, 256, 256), (128, 128, 100)], seed=42, qk_norm=False)
+    ctx, out, slots, _, _ = run_stack(B, wl, 0)
+    check(wl, out, stack_oracle(wl, rope=False))
+    ctx.close()
+
+
+def test_two_stream_block_large_model(B):
+    wl = dual_stack_workload(W.LARGE, "d", [(256, 256, 64), (128, 256, 0)], seed=43, qk_norm=True)
+    ctx, out, slots, _, _ = run_stack(B, wl, 3)
+    check(wl, out, stack_oracle(wl, rope=True))
+    ctx.close()
