@@ -111,11 +111,13 @@ def oracle_sample(wl: W.Workload):
     r = int(np.argmin(wl.token_lens))
     x = W.bf16_to_f64(wl.tokens[r])
     c = W.bf16_to_f64(wl.cond[r])
-    w0 = {k: W.bf16_to_f64(v) for k, v in wl.weights[0].items()}
+    w0 = {k: W.bf16_to_f64(v) for k, v in wl.weights[0].items() if k != "txt"}
+    if "txt" in wl.weights[0]:
+        w0["txt"] = {k: W.bf16_to_f64(v) for k, v in wl.weights[0]["txt"].items()}
+    req = wl.requests[r]
 
     def run():
-        return O.any_block_forward(x, c, w0, wl.dims.n_heads, wl.dims.ln_eps)
-    req = wl.requests[r]
+        return O.any_block_forward(x, c, w0, wl.dims.n_heads, wl.dims.ln_eps, n_img=req.n_image_tokens)
     desc = (f"request {r} of {wl.name} alone ({req.height}x{req.width}: {req.n_image_tokens} image + "
             f"{req.n_text_tokens} text tokens) through 1 of {wl.n_blocks} blocks, time scaled by {wl.n_blocks}; fp64 NumPy")
     return run, req.n_image_tokens / wl.n_blocks, desc
@@ -183,21 +185,28 @@ def run_gpu(args):
         par_rng = np.random.default_rng(args.seed + 3000)
         drawn = [W.draw_parallel_block_weights(par_rng, wl.dims) for _ in range(min(nb, 4))]
         wl.weights = [drawn[b % len(drawn)] for b in range(nb)]
+    if args.form == "dual":
+        txt_rng = np.random.default_rng(args.seed + 4000)
+        drawn = [W.draw_block_weights(txt_rng, wl.dims) for _ in range(min(nb, 2))]
+        wl.weights = [dict(w, txt=drawn[b % len(drawn)]) for b, w in enumerate(wl.weights)]
     if args.variants & 1:
         qk_rng = np.random.default_rng(args.seed + 2000)
-        wl.weights = [dict(w, **W.draw_qk_norm(qk_rng, wl.dims)) for w in wl.weights]
-    ctx = B.context_for(wl.dims, nb, wl.total_tokens, len(wl.requests), flags=args.variants)
-    B.upload_weights(ctx, wl.weights)
+        qk = W.draw_qk_norm(qk_rng, wl.dims)
+        wl.weights = [dict(w, **qk, **({"txt": dict(w["txt"], **qk)} if "txt" in w else {})) for w in wl.weights]
+    slots = nb * (2 if args.form == "dual" else 1)     # a two-stream block takes two weight slots
+    ctx = B.context_for(wl.dims, slots, wl.total_tokens, len(wl.requests), flags=args.variants)
+    assert B.upload_weights(ctx, wl.weights) == slots
     lens = wl.token_lens
     tok_bits, cond_bits = wl.packed_tokens(), wl.cond
     tok, cond = B.bits_to_cuda_bf16(tok_bits), B.bits_to_cuda_bf16(cond_bits)
     out = torch.empty((wl.total_tokens, wl.dims.hidden), dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
-    if args.variants:
-        # the rotary term needs each token's patch position: the step is given the requests themselves
-        step = lambda: ctx.dit_step_forward_requests(tok, wl.requests, cond, nb, out=out)
+    needs_geometry = bool(args.variants & 2) or args.form == "dual"
+    if args.variants or needs_geometry:
+        # the rotary term and two-stream blocks need each token's place in its request: the step is given the requests
+        step = lambda: ctx.dit_step_forward_requests(tok, wl.requests, cond, slots, out=out)
     else:
-        step = lambda: ctx.dit_step_forward(tok, lens, cond, nb, out=out)
+        step = lambda: ctx.dit_step_forward(tok, lens, cond, slots, out=out)
 
     def barrier():
         if dist is not None:
@@ -267,14 +276,14 @@ def run_gpu(args):
     e2e_steps = max(1, min(args.steps, 5))
 
     def e2e_step():
-        if args.variants & 2:     # the host-buffer entry point carries no geometry: copy, run, copy back by hand
+        if needs_geometry:        # the host-buffer entry point carries no geometry: copy, run, copy back by hand
             tok.copy_(h_tok.view(torch.bfloat16), non_blocking=True)
             cond.copy_(h_cond.view(torch.bfloat16), non_blocking=True)
             step()
             h_out.copy_(out, non_blocking=True)
             stream.synchronize()
         else:
-            ctx.dit_step_forward_host(h_tok, lens, h_cond, nb, h_out)
+            ctx.dit_step_forward_host(h_tok, lens, h_cond, slots, h_out)
 
     e2e_step()
     barrier()
@@ -310,7 +319,7 @@ def run_gpu(args):
         return max_over_ranks(e0.elapsed_time(e1)) / reps
 
     full_steps = max(1, min(args.steps, 5))
-    full_ms = timed_ms(lambda: ctx.dit_denoise_step(latents, text, wl.requests, dsig, pooled, nb), full_steps)
+    full_ms = timed_ms(lambda: ctx.dit_denoise_step(latents, text, wl.requests, dsig, pooled, slots), full_steps)
     full_launches = ctx.dit_last_launch_count()
     cond_dev = ctx.dit_timestep_cond(wl.requests, pooled)
     shell_ms = {"timestep_cond": timed_ms(lambda: ctx.dit_timestep_cond(wl.requests, pooled, cond_out=cond_dev), 5),
@@ -331,7 +340,7 @@ def run_gpu(args):
     per_launch_flops = {"gemm_qkv": 2.0 * T * H * 3 * H, "gemm_proj": 2.0 * T * H * H, "gemm_fc1": 2.0 * T * H * F,
                         "gemm_fc2": 2.0 * T * H * (F + (H if args.form == "parallel" else 0)),   # parallel form: one K = H + F output GEMM
                         "attention": 4.0 * H * sum(l * l for l in lens)}
-    per_launch_bytes = {"ln_modulate": T * H * (4 + 2), "modulation": nb * wl.dims.cond_dim * 6 * H * 2}
+    per_launch_bytes = {"ln_modulate": T * H * (4 + 2), "modulation": slots * wl.dims.cond_dim * 6 * H * 2}
     kern = {}
     for name, rec in kernels.items():
         if not rec["launches"]:
@@ -402,8 +411,9 @@ def main():
     ap.add_argument("--depth", type=int, default=0, help="run this many blocks instead of the configuration's (weights reused cyclically)")
     ap.add_argument("--variants", type=int, default=0, choices=[0, 1, 2, 3],
                     help="block variant bits: 1 = RMS-norm of queries and keys, 2 = 2-D rotary term (not the headline configuration)")
-    ap.add_argument("--form", default="sequential", choices=["sequential", "parallel"],
-                    help="block form: the adaLN-Zero block of the headline, or the parallel attention+MLP form (same FLOPs)")
+    ap.add_argument("--form", default="sequential", choices=["sequential", "parallel", "dual"],
+                    help="block form: the adaLN-Zero block of the headline, the parallel attention+MLP form, or the "
+                         "two-stream form with separate image/text tensors (same FLOPs each; not the headline)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":
