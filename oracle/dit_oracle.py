@@ -145,6 +145,31 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
     return out
 
 
+E4M3_MAX = 448.0
+
+
+def quantize_e4m3(x: np.ndarray) -> np.ndarray:
+    """Nearest value of the 8-bit float with 4 exponent and 3 mantissa bits (bias 7, no infinities,
+    largest finite value 448), ties to the even mantissa, larger magnitudes clamped to 448."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.abs(x)
+    _, e = np.frexp(a)                                  # a = m * 2^e, m in [0.5, 1)
+    step = np.exp2(np.maximum(e - 1, -6) - 3.0)         # spacing: 2^(exponent - 3), exponent >= -6 (subnormals)
+    q = np.minimum(np.rint(a / step) * step, E4M3_MAX)  # rint rounds halves to even
+    return np.sign(x) * q
+
+
+def fp8_linear(h: np.ndarray, w: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """h W + b with both operands reduced to e4m3: each row of h is scaled so that its largest
+    magnitude maps to 448, each column of W likewise; the product of the quantised operands is
+    exact and is scaled back."""
+    sa = np.abs(h).max(axis=1, keepdims=True) / E4M3_MAX
+    sw = np.abs(w).max(axis=0, keepdims=True) / E4M3_MAX
+    sa[sa == 0.0] = 1.0
+    sw[sw == 0.0] = 1.0
+    return (quantize_e4m3(h / sa) @ quantize_e4m3(w / sw)) * sa * sw + b
+
+
 def rms_norm_heads(z: np.ndarray, g: np.ndarray, n_heads: int, eps: float) -> np.ndarray:
     """RMS-norm of every head of every row: z_head / sqrt(mean(z_head^2) + eps) * g, g [d]."""
     L, H = z.shape
@@ -189,7 +214,7 @@ def patch_positions(height: int, width: int, n_text: int) -> np.ndarray:
 
 def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps: float,
                   rows: np.ndarray | None = None, taps: dict | None = None,
-                  positions: np.ndarray | None = None) -> np.ndarray:
+                  positions: np.ndarray | None = None, fp8: bool = False) -> np.ndarray:
     """One adaLN-Zero DiT block on one request.  x [L, H], cond [C] -> [L, H].
 
     With `rows`, only those output rows are produced (keys and values still
@@ -201,11 +226,15 @@ def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps
     ([d] each), queries and keys are RMS-normed per head (same eps) before
     attention; if `positions` [L, 2] is given, queries and keys then get the
     2-D rotary term.  The taps' qkv is taken after both.
+
+    With `fp8`, the two products that read a LayerNorm output (QKV and the MLP up-projection) take
+    their operands through fp8_linear; everything else is unchanged.
     """
     H = x.shape[1]
+    lin = fp8_linear if fp8 else (lambda a, ww, bb: a @ ww + bb)
     shift_a, scale_a, gate_a, shift_m, scale_m, gate_m = adaln_modulation(cond, w["w_ada"], w["b_ada"])
     h = modulate(layer_norm(x, eps), shift_a, scale_a)
-    qkv = h @ w["w_qkv"] + w["b_qkv"]
+    qkv = lin(h, w["w_qkv"], w["b_qkv"])
     q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
     if "q_norm" in w:
         q = rms_norm_heads(q, w["q_norm"], n_heads, eps)
@@ -218,7 +247,7 @@ def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps
     xr = x if rows is None else x[rows]
     x_mid = xr + gate_a * (a @ w["w_o"] + w["b_o"])
     h2 = modulate(layer_norm(x_mid, eps), shift_m, scale_m)
-    u = gelu_tanh(h2 @ w["w_fc1"] + w["b_fc1"])
+    u = gelu_tanh(lin(h2, w["w_fc1"], w["b_fc1"]))
     y = x_mid + gate_m * (u @ w["w_fc2"] + w["b_fc2"])
     if taps is not None:
         taps.update(h1=h, qkv=qkv, a=a, x_mid=x_mid, h2=h2, u=u)
@@ -227,7 +256,7 @@ def block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps
 
 def parallel_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads: int, eps: float,
                            rows: np.ndarray | None = None, taps: dict | None = None,
-                           positions: np.ndarray | None = None) -> np.ndarray:
+                           positions: np.ndarray | None = None, fp8: bool = False) -> np.ndarray:
     """The parallel (single-modulation) form of the block: attention and the MLP read the same
     modulated LayerNorm output, their results are concatenated and share one output projection:
 
@@ -239,9 +268,10 @@ def parallel_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads:
     Optional q_norm / k_norm and `positions` act on queries and keys as in block_forward.
     """
     H = x.shape[1]
+    lin = fp8_linear if fp8 else (lambda a, ww, bb: a @ ww + bb)
     shift, scale, gate = np.split(silu(cond) @ w["w_ada"] + w["b_ada"], 3)
     h = modulate(layer_norm(x, eps), shift, scale)
-    qkv = h @ w["w_qkv"] + w["b_qkv"]
+    qkv = lin(h, w["w_qkv"], w["b_qkv"])
     q, k, v = qkv[:, :H], qkv[:, H:2 * H], qkv[:, 2 * H:]
     if "q_norm" in w:
         q = rms_norm_heads(q, w["q_norm"], n_heads, eps)
@@ -250,7 +280,7 @@ def parallel_block_forward(x: np.ndarray, cond: np.ndarray, w: Weights, n_heads:
         q, k = rope_2d(q, positions, n_heads), rope_2d(k, positions, n_heads)
     a = attention(q, k, v, n_heads, rows)
     hr, xr = (h, x) if rows is None else (h[rows], x[rows])
-    u = gelu_tanh(hr @ w["w_fc1"] + w["b_fc1"])
+    u = gelu_tanh(lin(hr, w["w_fc1"], w["b_fc1"]))
     y = xr + gate * (np.concatenate([a, u], axis=1) @ w["w_out"] + w["b_out"])
     if taps is not None:
         taps.update(h1=h, qkv=np.concatenate([q, k, v], axis=1), a=a, u=u)
@@ -304,24 +334,25 @@ def any_block_forward(x, cond, w: Weights, n_heads: int, eps: float, n_img: int 
 
 def stack_forward_alone(x: np.ndarray, cond: np.ndarray, blocks: Sequence[Weights],
                         n_heads: int, eps: float, positions: np.ndarray | None = None,
-                        n_img: int | None = None) -> np.ndarray:
-    """A stack of blocks on one request run by itself."""
+                        n_img: int | None = None, fp8: bool = False) -> np.ndarray:
+    """A stack of blocks on one request run by itself (fp8: sequential and parallel forms only)."""
     for w in blocks:
-        x = any_block_forward(x, cond, w, n_heads, eps, n_img=n_img, positions=positions)
+        kw = {"fp8": True} if fp8 else {}
+        x = any_block_forward(x, cond, w, n_heads, eps, n_img=n_img, positions=positions, **kw)
     return x
 
 
 def step_forward(packed: np.ndarray, token_lens: Sequence[int], cond: np.ndarray,
                  blocks: Sequence[Weights], n_heads: int, eps: float,
                  positions: Sequence[np.ndarray] | None = None,
-                 n_imgs: Sequence[int] | None = None) -> np.ndarray:
+                 n_imgs: Sequence[int] | None = None, fp8: bool = False) -> np.ndarray:
     """One denoising step over a packed batch: each request through the stack on its own."""
     out = np.empty_like(packed)
     p = 0
     for r, l in enumerate(token_lens):
         out[p:p + l] = stack_forward_alone(packed[p:p + l], cond[r], blocks, n_heads, eps,
                                            None if positions is None else positions[r],
-                                           None if n_imgs is None else n_imgs[r])
+                                           None if n_imgs is None else n_imgs[r], fp8)
         p += l
     return out
 

@@ -245,3 +245,58 @@ def test_dual_block_streams_meet_only_in_attention():
     # row subset and stack dispatch
     assert np.array_equal(O.dual_block_forward(x, cond, dual, n_img, heads, 1e-6, rows=np.array([5, 0])), y[[5, 0]])
     assert np.array_equal(O.stack_forward_alone(x, cond, [dual], heads, 1e-6, n_img=n_img), y)
+
+
+# ----------------------------------------------------------------------------- fp8 (e4m3) operands
+def test_e4m3_grid():
+    q = O.quantize_e4m3
+    # representable values stay as they are, both signs
+    vals = np.array([0.0, 2.0 ** -9, 2.0 ** -6, 0.875 * 2.0 ** -6, 1.0, 1.125, 1.875, 240.0, 448.0, -3.5, -0.0625])
+    assert np.array_equal(q(vals), vals)
+    # ties go to the even mantissa; everything beyond 448 is clamped
+    assert q(1.0625) == 1.0 and q(1.1875) == 1.25 and q(1.0626) == 1.125
+    assert q(2.0 ** -10) == 0.0 and q(3 * 2.0 ** -10) == 2.0 ** -8 and q(2.0 ** -10 * 1.01) == 2.0 ** -9
+    assert q(464.0) == 448.0 and q(1e6) == 448.0 and q(-1e6) == -448.0 and q(447.0) == 448.0 and q(431.0) == 416.0
+    # the format has 126 positive finite values: 7 subnormals and 15 binades of 8 values, less the NaN code
+    grid = np.unique(q(np.linspace(0.0, 500.0, 2_000_001)))
+    sub = np.unique(q(np.linspace(0.0, 2.0 ** -6, 100_001)))
+    assert len(np.union1d(grid, sub)) - 1 == 126
+    # relative error of a normal value is at most 2^-4
+    x = np.exp(np.random.default_rng(0).uniform(np.log(2.0 ** -6), np.log(448.0), 10000))
+    assert (np.abs(q(x) - x) / x).max() <= 2.0 ** -4
+
+
+def test_fp8_linear_is_exact_on_grid_operands_and_close_otherwise():
+    rng = np.random.default_rng(1)
+    # operands already on the e4m3 grid with row / column maxima of 448: nothing is lost
+    h = O.quantize_e4m3(rng.uniform(-448, 448, (5, 16))); h[:, 0] = 448.0
+    w = O.quantize_e4m3(rng.uniform(-448, 448, (16, 7))); w[0, :] = -448.0
+    b = rng.standard_normal(7)
+    assert np.allclose(O.fp8_linear(h, w, b), h @ w + b, rtol=1e-14)
+    # scaling a row of h or a column of W scales the same row / column of the product exactly
+    # (powers of two keep the quantised mantissas)
+    h2, w2 = rng.standard_normal((6, 64)), rng.standard_normal((64, 9)) * 0.02
+    base = O.fp8_linear(h2, w2, np.zeros(9))
+    hs = h2.copy(); hs[2] *= 8.0
+    ws = w2.copy(); ws[:, 4] *= 0.25
+    assert np.array_equal(O.fp8_linear(hs, w2, np.zeros(9))[2], base[2] * 8.0)
+    assert np.array_equal(O.fp8_linear(h2, ws, np.zeros(9))[:, 4], base[:, 4] * 0.25)
+    # and the result is a few per cent from the exact product
+    exact = h2 @ w2
+    assert 1e-3 < O.error_metric(base, exact) < 0.3
+    # zero rows and columns do not divide by zero
+    hz = h2.copy(); hz[1] = 0.0
+    assert np.isfinite(O.fp8_linear(hz, w2, np.zeros(9))).all()
+
+
+def test_fp8_block_is_the_plain_block_with_two_products_swapped():
+    rng = np.random.default_rng(2)
+    H, F, C, heads, L = 64, 128, 8, 2, 5
+    w = _block(rng, H, F, C)
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    taps8, taps = {}, {}
+    y8 = O.block_forward(x, cond, w, heads, 1e-6, taps=taps8, fp8=True)
+    y = O.block_forward(x, cond, w, heads, 1e-6, taps=taps)
+    assert np.array_equal(taps8["h1"], taps["h1"])                          # LayerNorm is untouched
+    assert np.array_equal(taps8["qkv"], O.fp8_linear(taps["h1"], w["w_qkv"], w["b_qkv"]))
+    assert 1e-4 < O.error_metric(y8, y) < 0.2
