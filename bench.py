@@ -379,9 +379,10 @@ def run_gpu(args):
            "seconds_per_sample": cpu_s, "repeats": reps}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16+e4m3 (reduced precision, not the headline)" if args.variants & 4 else "f16",
             "data": "synthetic",
-            "config": {"workload": wl.name, "block_form": args.form, "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2)}, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
+            "config": {"workload": wl.name, "block_form": args.form, "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2), "fp8_qkv_fc1": bool(args.variants & 4)}, "n_blocks": nb, "weights_reused_cyclically": bool(args.depth), "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
                        "total_tokens": T, "image_tokens": wl.image_tokens, "hidden": H, "heads": wl.dims.n_heads,
                        "head_dim": wl.dims.head_dim, "mlp_hidden": F, "parallelism": f"replicas x{world}",
                        "l2": "weights and activations of a step exceed L2 (126 MB); no flush"},
@@ -409,8 +410,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0, help="run this many blocks instead of the configuration's (weights reused cyclically)")
-    ap.add_argument("--variants", type=int, default=0, choices=[0, 1, 2, 3],
-                    help="block variant bits: 1 = RMS-norm of queries and keys, 2 = 2-D rotary term (not the headline configuration)")
+    ap.add_argument("--variants", type=int, default=0, choices=list(range(8)),
+                    help="context flag bits: 1 = RMS-norm of queries and keys, 2 = 2-D rotary term, 4 = e4m3 operands for the "
+                         "QKV and up-projection GEMMs (reduced precision: never the headline configuration)")
     ap.add_argument("--form", default="sequential", choices=["sequential", "parallel", "dual"],
                     help="block form: the adaLN-Zero block of the headline, the parallel attention+MLP form, or the "
                          "two-stream form with separate image/text tensors (same FLOPs each; not the headline)")

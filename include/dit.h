@@ -82,6 +82,13 @@ typedef struct {
  *                        or dit_denoise_step (dit_step_forward returns DIT_ERR_INVALID_ARG). */
 #define DIT_FLAG_QK_RMSNORM 1u
 #define DIT_FLAG_ROPE_2D 2u
+/* Reduced-precision mode, off in every benchmark configuration: the two GEMMs that read a LayerNorm
+ * output (QKV projection and MLP up-projection, 7/12 of a block's linear FLOPs) take e4m3 operands.
+ * Each row of the modulated LayerNorm output is scaled so that its largest magnitude maps to 448 and
+ * rounded to e4m3 by the LayerNorm kernel; each output channel of W_qkv / W_fc1 likewise at load time;
+ * the accumulator (fp32, exact products) is scaled back in the epilogue.  Everything else stays as
+ * it is.  Errors grow to a few per cent of the output's rms; not available for two-stream blocks. */
+#define DIT_FLAG_FP8_GEMM 4u
 
 /* One request of the paper's problem statement (Section 3): an image resolution, a position in
  * its denoising schedule and the diffusion time of this step.  Image tokens = (height/16) *

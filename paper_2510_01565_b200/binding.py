@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(HERE, "libdit.so")
 DIT_OK = 0
 DIT_FLAG_QK_RMSNORM = 1
 DIT_FLAG_ROPE_2D = 2
+DIT_FLAG_FP8_GEMM = 4
 STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
                 "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
 KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]

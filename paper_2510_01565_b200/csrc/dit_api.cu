@@ -28,7 +28,9 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets (bytes) inside one block's weight slot.
 struct BlockLayout {
-  size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, q_norm, k_norm, bytes;
+  size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, q_norm, k_norm;
+  size_t s_qkv, s_fc1;   // per-output-channel scales of the e4m3 weights (DIT_FLAG_FP8_GEMM)
+  size_t bytes;
 };
 // Offsets (bytes) inside the workspace.
 struct Layout {
@@ -38,6 +40,7 @@ struct Layout {
   size_t sh_w_in, sh_b_in, sh_w_t1, sh_b_t1, sh_w_t2, sh_b_t2, sh_w_fa, sh_b_fa, sh_w_out, sh_b_out;
   size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok;
   size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
+  size_t row_scale;    // per-row scales of the e4m3 activations (DIT_FLAG_FP8_GEMM)
   size_t items;        // two-stream launches: [0] item count, then per-tile flags, then the items
   size_t bytes;
 };
@@ -52,7 +55,7 @@ bool config_ok(const dit_config* c) {
   if (c->cond_dim < 1 || c->cond_dim > kMaxCondDim) return false;
   if (c->max_blocks < 1 || c->max_total_tokens < 1) return false;
   if (c->max_requests < 1 || c->max_requests > DIT_MAX_REQUESTS) return false;
-  if (!(c->ln_eps >= 0.f) || (c->flags & ~static_cast<uint32_t>(DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D))) return false;
+  if (!(c->ln_eps >= 0.f) || (c->flags & ~static_cast<uint32_t>(DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D | DIT_FLAG_FP8_GEMM))) return false;
   return true;
 }
 
@@ -75,6 +78,8 @@ Layout make_layout(const dit_config& c) {
   L.blk.b_fc2 = take(H * 4);
   L.blk.q_norm = take(c.head_dim * 4);
   L.blk.k_norm = take(c.head_dim * 4);
+  L.blk.s_qkv = take(3 * H * 4);
+  L.blk.s_fc1 = take(F * 4);
   L.blk.bytes = o;
   o = 0;
   L.weights = take(L.blk.bytes * c.max_blocks);
@@ -104,6 +109,7 @@ Layout make_layout(const dit_config& c) {
   L.sh_modfin = take(R * 2 * H * 4);
   L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
   L.rope_theta = take(64 * 4);
+  L.row_scale = take(T * 4);
   L.items = take((16 + 3 * (T / (2 * 128) + 2)) * 4);
   L.bytes = o;
   return L;
@@ -169,6 +175,18 @@ bool make_map(const dit_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t inne
   return r == CUDA_SUCCESS;
 }
 
+// The same for e4m3 operands: 1 byte per element, box 128 bytes x box_rows.
+bool make_map8(const dit_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner};
+  cuuint32_t box[2] = {128, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
   s->n = n;
   s->cu[0] = 0;
@@ -184,17 +202,17 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
 
 const RowGeom kNoGeom{};
 
-template <int EPI, int HD = 0, bool DUAL = false>
+template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                         const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom, const CUtensorMap* tmB2 = nullptr) {
   // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
   GemmParams q = p;
-  const long long band_bytes = 2ll * gemm_cfg::BM * p.K * 2;
+  const long long band_bytes = 2ll * gemm_cfg::BM * p.K * (FP8 ? 1 : 2);
   q.band = static_cast<int>(std::max(1ll, std::min<long long>((36ll << 20) / band_bytes, (p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM))));
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);   // a two-stream launch may have more items than row tiles: the loop covers them
-  gemm_tcgen05_kernel<EPI, HD, DUAL><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
+  gemm_tcgen05_kernel<EPI, HD, DUAL, FP8><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
   return cudaGetLastError();
 }
 
@@ -207,14 +225,14 @@ cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, cons
 }
 
 // LayerNorm + modulate launch: picks the register-resident row width (float4 per lane) for H.
-template <bool kFromBf16>
+template <bool kFromBf16, bool kOutFp8 = false>
 cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
                       long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st,
-                      long long kind_stride = 0, const RowGeom& geo = kNoGeom) {
+                      long long kind_stride = 0, const RowGeom& geo = kNoGeom, float* row_scale = nullptr) {
   const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
-  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
-  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
-  else ln_modulate_kernel<kFromBf16, 32><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo);
+  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
+  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
+  else ln_modulate_kernel<kFromBf16, 32, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
   return cudaGetLastError();
 }
 
@@ -229,6 +247,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   SeqInfo seq{};
   if (!build_seq(lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
   const bool qk_variant = (c.flags & (DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D)) != 0;
+  const bool fp8 = (c.flags & DIT_FLAG_FP8_GEMM) != 0;     // QKV and up-projection read e4m3 h and weights
   if ((c.flags & DIT_FLAG_ROPE_2D) && !geo)
     return fail(ctx, DIT_ERR_INVALID_ARG, "the rotary term needs the requests' geometry: use dit_step_forward_requests");
   const int T = seq.total, H = c.hidden, F = c.mlp_hidden;
@@ -251,6 +270,9 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM) || !make_map(ctx, &tm_a, a, H, T, gemm_cfg::BM) ||
       !make_map(ctx, &tm_u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &tm_qkv, qkv, 3 * H, T, 128) ||
       !make_map(ctx, &tm_cat, cat, H + F, T, gemm_cfg::BM))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  float* row_scale = ctx->at<float>(ctx->lay.row_scale);
+  if (fp8 && !make_map8(ctx, &tm_h, h, H, T, gemm_cfg::BM))   // h holds e4m3 codes in this mode
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
 
   int64_t launches = 0;
@@ -331,6 +353,9 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     };
     // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
+      if (fp8)
+        return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale)
+                      : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale);
       return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg)
                     : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
     }));
@@ -341,6 +366,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_qkv);
     g.out16 = qkv;
     two_stream(g, ctx->lay.blk.b_qkv);
+    if (fp8) { g.row_scale = row_scale; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_qkv); }
     if (qk_variant) {
       g.hidden = H; g.eps = c.ln_eps;
       if (c.flags & DIT_FLAG_QK_RMSNORM) {
@@ -351,6 +377,9 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       }
       if (c.flags & DIT_FLAG_ROPE_2D) g.rope_theta = ctx->at<float>(ctx->lay.rope_theta);
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+        if (fp8)
+          return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg)
+                                   : launch_gemm<kEpiQkvF16, 64, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg);
         if (dual)
           return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
                                    : launch_gemm<kEpiQkvF16, 64, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv);
@@ -359,6 +388,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       }));
     } else {
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+        if (fp8) return launch_gemm<kEpiBiasF16, 0, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st);
         return dual ? launch_gemm<kEpiBiasF16, 0, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
                     : launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st);
       }));
@@ -381,7 +411,11 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       g.M = T; g.N = F; g.K = H;
       g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
       g.out16 = cat + H; g.ld16 = H + F;
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st); }));
+      if (fp8) { g.row_scale = row_scale; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc1); }
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
+        return fp8 ? launch_gemm<kEpiBiasGeluF16, 0, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st)
+                   : launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st);
+      }));
       // one output projection over [attention | MLP] + gate + residual
       g = GemmParams{};
       g.status = status;
@@ -406,7 +440,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }));
     // LN2 + modulate
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      return launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
+      return fp8 ? launch_ln<false, true>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale)
+                 : launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
     }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};
@@ -415,7 +450,9 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
     g.out16 = u;
     two_stream(g, ctx->lay.blk.b_fc1);
+    if (fp8) { g.row_scale = row_scale; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc1); }
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
+      if (fp8) return launch_gemm<kEpiBiasGeluF16, 0, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st);
       return dual ? launch_gemm<kEpiBiasGeluF16, 0, true>(ctx, tm_h, bs.tm_fc1, g, seq, st, rg, &bt.tm_fc1)
                   : launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st);
     }));
@@ -529,6 +566,10 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32, 0, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16, 0, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16, 0, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>), mod_smem_bytes(kMaxCondDim));  // same for every context
@@ -591,21 +632,28 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
     transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
     return cudaGetLastError();
   };
+  const bool fp8 = (ctx->cfg.flags & DIT_FLAG_FP8_GEMM) != 0;
+  auto weight8 = [&](const void* src, size_t off, size_t scale_off, int K, int N) {   // [K, N] bf16 -> e4m3 [N, K] + scales [N]
+    col_absmax_scale_kernel<<<(N + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + scale_off), K, N);
+    dim3 grid((N + 31) / 32, (K + 31) / 32);
+    transpose_bf16_to_e4m3_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<const float*>(base + scale_off), base + off, K, N);
+    return cudaGetLastError();
+  };
   DIT_CUDA_TRY(ctx, bias(w->b_ada, L.b_ada, 6 * H));
-  DIT_CUDA_TRY(ctx, weight(w->w_qkv, L.w_qkv, H, 3 * H));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_qkv, L.w_qkv, L.s_qkv, H, 3 * H) : weight(w->w_qkv, L.w_qkv, H, 3 * H));
   DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
   DIT_CUDA_TRY(ctx, weight(w->w_o, L.w_o, H, H));
   DIT_CUDA_TRY(ctx, bias(w->b_o, L.b_o, H));
-  DIT_CUDA_TRY(ctx, weight(w->w_fc1, L.w_fc1, H, F));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_fc1, L.w_fc1, L.s_fc1, H, F) : weight(w->w_fc1, L.w_fc1, H, F));
   DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
   DIT_CUDA_TRY(ctx, weight(w->w_fc2, L.w_fc2, F, H));
   DIT_CUDA_TRY(ctx, bias(w->b_fc2, L.b_fc2, H));
   DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));   // NULL scale = ones
   DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
 
-  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) ||
+  if (!(fp8 ? make_map8(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2)) ||
       !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) ||
-      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) ||
+      !(fp8 ? make_map8(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2)) ||
       !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;
@@ -617,6 +665,7 @@ dit_status dit_load_dual_block_weights(dit_ctx* ctx, int32_t b, const dit_block_
   if (!ctx) return DIT_ERR_INVALID_ARG;
   ctx->err[0] = 0;
   if (b < 0 || b + 1 >= ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "a two-stream block needs slots b and b + 1 inside [0, max_blocks)");
+  if (ctx->cfg.flags & DIT_FLAG_FP8_GEMM) return fail(ctx, DIT_ERR_SHAPE, "two-stream blocks are not available with DIT_FLAG_FP8_GEMM");
   dit_status s = dit_load_block_weights(ctx, b, image_stream, stream);
   if (s != DIT_OK) return s;
   s = dit_load_block_weights(ctx, b + 1, text_stream, stream);
@@ -656,17 +705,24 @@ dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_pa
     return cudaGetLastError();
   };
   DIT_CUDA_TRY(ctx, cudaMemsetAsync(base + L.b_ada, 0, static_cast<size_t>(6) * H * 4, st));
+  const bool fp8 = (ctx->cfg.flags & DIT_FLAG_FP8_GEMM) != 0;
+  auto weight8 = [&](const void* src, size_t off, size_t scale_off, int K, int N) {   // [K, N] bf16 -> e4m3 [N, K] + scales [N]
+    col_absmax_scale_kernel<<<(N + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<float*>(base + scale_off), K, N);
+    dim3 grid((N + 31) / 32, (K + 31) / 32);
+    transpose_bf16_to_e4m3_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<const float*>(base + scale_off), base + off, K, N);
+    return cudaGetLastError();
+  };
   DIT_CUDA_TRY(ctx, bias(w->b_ada, L.b_ada, 3 * H));
-  DIT_CUDA_TRY(ctx, weight(w->w_qkv, L.w_qkv, H, 3 * H));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_qkv, L.w_qkv, L.s_qkv, H, 3 * H) : weight(w->w_qkv, L.w_qkv, H, 3 * H));
   DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
-  DIT_CUDA_TRY(ctx, weight(w->w_fc1, L.w_fc1, H, F));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_fc1, L.w_fc1, L.s_fc1, H, F) : weight(w->w_fc1, L.w_fc1, H, F));
   DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
   DIT_CUDA_TRY(ctx, weight(w->w_out, L.w_o, H + F, H));          // runs on over the W_fc2 region
   DIT_CUDA_TRY(ctx, bias(w->b_out, L.b_fc2, H));
   DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));
   DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
-  if (!make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) ||
-      !make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) ||
+  if (!(fp8 ? make_map8(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2)) ||
+      !(fp8 ? make_map8(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2)) ||
       !make_map(ctx, &bs.tm_fc2, base + L.w_o, H + F, H, gemm_cfg::BN / 2))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;

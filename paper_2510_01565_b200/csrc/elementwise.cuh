@@ -140,12 +140,14 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 // ------------------------------------------------------------------------------------------------
 constexpr int kLnWarps = 4;
 
-template <bool kFromBf16, int kLnMaxVec>
+// kOutFp8: h is written as e4m3 codes (1 byte per element, `h` then points at bytes) with one scale per
+// row, largest magnitude of the row -> 448; the scale goes to row_scale[row].
+template <bool kFromBf16, int kLnMaxVec, bool kOutFp8 = false>
 __global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVec <= 24 ? 4 : 3)))
 ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
                    const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                    int T, int H, float eps, const __grid_constant__ SeqInfo seq,
-                   long long kind_stride, const __grid_constant__ RowGeom geo) {
+                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale) {
   const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= T) return;
@@ -186,6 +188,36 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
   const long long voff = req * req_stride + (kind_stride ? row_kind(seq, geo, req, row) * kind_stride : 0);
   const float4* sh = reinterpret_cast<const float4*>(shift0 + voff);
   const float4* sc = reinterpret_cast<const float4*>(scale0 + voff);
+  if (kOutFp8) {
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < kLnMaxVec; ++i) {
+      const int idx = i * 32 + lane;
+      if (idx < nvec) {
+        const float4 s1 = __ldg(sc + idx), s0 = __ldg(sh + idx);
+        v[i].x = (v[i].x - mean) * rstd * (1.f + s1.x) + s0.x;
+        v[i].y = (v[i].y - mean) * rstd * (1.f + s1.y) + s0.y;
+        v[i].z = (v[i].z - mean) * rstd * (1.f + s1.z) + s0.z;
+        v[i].w = (v[i].w - mean) * rstd * (1.f + s1.w) + s0.w;
+        amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
+    if (lane == 0) row_scale[row] = amax > 0.f ? amax / 448.0f : 1.0f;
+    uint32_t* dst8 = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(h) + static_cast<size_t>(row) * H);
+#pragma unroll
+    for (int i = 0; i < kLnMaxVec; ++i) {
+      const int idx = i * 32 + lane;
+      if (idx < nvec) {
+        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[i].x * inv, v[i].y * inv), __NV_SATFINITE, __NV_E4M3);
+        const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v[i].z * inv, v[i].w * inv), __NV_SATFINITE, __NV_E4M3);
+        dst8[idx] = lo | (hi << 16);
+      }
+    }
+    return;
+  }
   uint2* dst = reinterpret_cast<uint2*>(h + static_cast<size_t>(row) * H);
 #pragma unroll
   for (int i = 0; i < kLnMaxVec; ++i) {
@@ -270,6 +302,37 @@ transpose_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __res
 }
 
 // Widens a bf16 vector to fp32; a NULL input stands for a constant vector of `fill`.
+// ------------------------------------------------------------------------------------------------
+// FP8 weight load: per output channel n, scale[n] = max_k |W[k, n]| / 448, then
+// bf16 [K, N] row-major -> e4m3 [N, K] row-major of W[k, n] / scale[n].
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+col_absmax_scale_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ scale, int K, int N) {
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= N) return;
+  float amax = 0.f;
+  for (int k = 0; k < K; ++k) amax = fmaxf(amax, fabsf(__bfloat162float(in[static_cast<size_t>(k) * N + n])));
+  scale[n] = amax > 0.f ? amax / 448.0f : 1.0f;
+}
+
+__global__ void __launch_bounds__(256)
+transpose_bf16_to_e4m3_kernel(const __nv_bfloat16* __restrict__ in, const float* __restrict__ scale,
+                              uint8_t* __restrict__ out, int K, int N) {
+  __shared__ float tile[32][33];
+  const int n0 = blockIdx.x * 32, k0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+  for (int i = ty; i < 32; i += 8) {
+    const int k = k0 + i, n = n0 + tx;
+    tile[i][tx] = (k < K && n < N) ? __bfloat162float(in[static_cast<size_t>(k) * N + n]) : 0.f;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int n = n0 + i, k = k0 + tx;
+    if (n < N && k < K)
+      out[static_cast<size_t>(n) * K + k] = static_cast<uint8_t>(__nv_cvt_float_to_fp8(tile[tx][i] / scale[n], __NV_SATFINITE, __NV_E4M3));
+  }
+}
+
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, int n, float fill) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = in ? __bfloat162float(in[i]) : fill;

@@ -54,6 +54,9 @@ struct GemmParams {
   const float* q_norm2;
   const float* k_norm2;
   long long gate_kind_stride;   // text stream's gate vector = gate + gate_kind_stride
+  // FP8 launches only: A and Wt hold e4m3 codes; out = acc * row_scale[m] * col_scale[n] + bias
+  const float* row_scale;   // [M]
+  const float* col_scale;   // [N]
 };
 
 namespace gemm_cfg {
@@ -89,7 +92,9 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int ban
 // DUAL: two-stream launch.  The weight operand comes from tmB for image-token rows and from tmB2 for
 // text-token rows; the row tiles to visit are listed in p.items (built on the device from the batch's
 // geometry), everything else is unchanged.
-template <int EPI, int HD = 0, bool DUAL = false>
+// FP8: both operands are e4m3 (1 byte per element, 128 elements per 128-byte swizzled row, K = 32
+// per MMA); the row and column scales that map the codes back are applied in the epilogue.
+template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmB2, const GemmParams p,
@@ -121,7 +126,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (DUAL) { const int it = __ldg(p.items + ib); mb = it & 0xFFFFFF; kind = it >> 24; }
     else { mb = ib; kind = 0; }
   };
-  const int num_k = (p.K + BK - 1) / BK;
+  constexpr int BKE = FP8 ? 2 * BK : BK;                      // elements of K per stage (128 bytes per row)
+  const int num_k = (p.K + BKE - 1) / BKE;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -153,8 +159,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t full_leader = map_to_cta(full_bar(stage), 0);
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE_BYTES);   // both CTAs' bytes
           const uint32_t sa = base + stage * STAGE_BYTES;
-          tma_load_2d_pair(sa, &tmA, kb * BK, m0, full_leader);
-          tma_load_2d_pair(sa + A_BYTES, tb, kb * BK, n0, full_leader);
+          tma_load_2d_pair(sa, &tmA, kb * BKE, m0, full_leader);
+          tma_load_2d_pair(sa + A_BYTES, tb, kb * BKE, n0, full_leader);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -162,7 +168,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = idesc_f16(2 * BM, BN, false);
+      constexpr uint32_t idesc = FP8 ? idesc_e4m3(2 * BM, BN) : idesc_f16(2 * BM, BN, false);
       int stage = 0; uint32_t phase = 0; int it = 0;
       for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
         const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
@@ -176,8 +182,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint64_t adesc = smem_desc_sw128(sa, 16, 1024);
           const uint64_t bdesc = smem_desc_sw128(sa + A_BYTES, 16, 1024);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)   // 32 bytes further along K inside the swizzled row
-            umma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          for (int k = 0; k < BK / 16; ++k) { // 32 bytes further along K inside the swizzled row
+            if (FP8) umma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            else umma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          }
           umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -203,6 +211,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int my_kind = -1;
       if (DUAL && row < p.M) my_kind = row_kind(seq, geo, my_req, row);
       const bool row_ok = row < p.M && (!DUAL || my_kind == kind);
+      const float sa = (FP8 && row < p.M) ? p.row_scale[row] : 1.0f;
       const float* bias = (DUAL && kind) ? p.bias2 : p.bias;
       const float* gate = p.gate + ((DUAL && kind) ? p.gate_kind_stride : 0);
       const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
@@ -246,7 +255,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             tmem_ld32(t_row + hc * HD + q * 32, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[q * 32 + i] = __uint_as_float(r[i]) + __ldg(bias + colh + q * 32 + i);
+            for (int i = 0; i < 32; ++i) {
+              float acc_v = __uint_as_float(r[i]);
+              if (FP8) acc_v *= sa * __ldg(p.col_scale + colh + q * 32 + i);
+              v[q * 32 + i] = acc_v + __ldg(bias + colh + q * 32 + i);
+            }
           }
           if (row_ok) {
             const int part = colh / p.hidden;  // 0 = Q, 1 = K, 2 = V
@@ -352,8 +365,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
                 const int i = 8 * v + 2 * h;
-                float a = __uint_as_float(r[i]) + __ldg(bias + col0 + i);
-                float b = __uint_as_float(r[i + 1]) + __ldg(bias + col0 + i + 1);
+                float a = __uint_as_float(r[i]), b = __uint_as_float(r[i + 1]);
+                if (FP8) { a *= sa * __ldg(p.col_scale + col0 + i); b *= sa * __ldg(p.col_scale + col0 + i + 1); }
+                a += __ldg(bias + col0 + i);
+                b += __ldg(bias + col0 + i + 1);
                 if (EPI == kEpiBiasGeluF16) { a = gelu_tanh_f32(a); b = gelu_tanh_f32(b); }
                 const __half2 hh = __floats2half2_rn(a, b);
                 w[h] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -364,7 +379,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               if (col0 + i < p.N) {
-                float a = __uint_as_float(r[i]) + bias[col0 + i];
+                float a = __uint_as_float(r[i]);
+                if (FP8) a *= sa * p.col_scale[col0 + i];
+                a += bias[col0 + i];
                 if (EPI == kEpiBiasGeluF16) a = gelu_tanh_f32(a);
                 dst[i] = __float2half_rn(a);
               }

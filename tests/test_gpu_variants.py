@@ -305,3 +305,60 @@ def test_two_stream_block_large_model(B):
     ctx, out, slots, _, _ = run_stack(B, wl, 3)
     check(wl, out, stack_oracle(wl, rope=True))
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- fp8 (e4m3) operands
+# e4m3 keeps 3 mantissa bits, so this mode has its own, looser bar, stated per request as
+# rms(gpu - oracle) / rms(oracle):  <= 1e-1 against the exact oracle, and <= 2e-2 against the oracle that
+# quantises the same operands the same way (what is left there are codes that fall on the other side
+# of a rounding boundary in fp32 and in fp64, one e4m3 step each).  The largest single deviation is
+# checked too, against the quantising oracle only.
+FP8_RMS_EXACT = 1e-1
+FP8_RMS_QUANTISED = 2e-2
+FP8_MAX_QUANTISED = 2.5e-1
+
+
+def fp8_oracle(wl, rope, fp8):
+    pos = [O.patch_positions(q.height, q.width, q.n_text_tokens) for q in wl.requests] if rope else None
+    return O.step_forward(W.bf16_to_f64(wl.packed_tokens()), wl.token_lens, W.bf16_to_f64(wl.cond), f64_blocks(wl),
+                          wl.dims.n_heads, wl.dims.ln_eps, positions=pos, fp8=fp8)
+
+
+def worst_errors(wl, out, ref):
+    """(largest max|d|/rms, largest rms(d)/rms) over the requests."""
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    p, worst_max, worst_rms = 0, 0.0, 0.0
+    for l in wl.token_lens:
+        d, r = got[p:p + l] - ref[p:p + l], np.sqrt((ref[p:p + l] ** 2).mean())
+        worst_max, worst_rms = max(worst_max, np.abs(d).max() / r), max(worst_rms, np.sqrt((d ** 2).mean()) / r)
+        p += l
+    return worst_max, worst_rms
+
+
+def check_fp8(wl, out, rope):
+    q_max, q_rms = worst_errors(wl, out, fp8_oracle(wl, rope, fp8=True))
+    _, x_rms = worst_errors(wl, out, fp8_oracle(wl, rope, fp8=False))
+    assert q_rms <= FP8_RMS_QUANTISED and q_max <= FP8_MAX_QUANTISED, f"against the quantising oracle: rms {q_rms:.3e}, max {q_max:.3e}"
+    assert x_rms <= FP8_RMS_EXACT, f"against the exact oracle: rms {x_rms:.3e}"
+    assert q_rms < 0.5 * x_rms, "the result should follow the quantising oracle, not the exact one"
+
+
+@pytest.mark.parametrize("flags", [4, 7])
+def test_fp8_gemms_small_model(B, flags):
+    wl = dual_stack_workload(W.SMALL, "sps", MIXED, seed=51, qk_norm=bool(flags & 1))
+    ctx, out, slots, tok, cond = run_stack(B, wl, flags)
+    check_fp8(wl, out, bool(flags & 2))
+    ctx.close()
+
+
+def test_fp8_gemms_large_model_and_refusals(B):
+    wl = dual_stack_workload(W.LARGE, "sp", [(256, 256, 64), (128, 256, 0)], seed=52, qk_norm=False)
+    ctx, out, slots, tok, cond = run_stack(B, wl, 4)
+    check_fp8(wl, out, False)
+    # two-stream blocks are refused in this mode
+    dual = dual_stack_workload(W.LARGE, "d", [(256, 256, 64)], seed=53, qk_norm=False)
+    with pytest.raises(B.DitError) as e:
+        B.upload_weights(ctx, dual.weights)
+    assert e.value.status == 2
+    ctx.close()
