@@ -48,10 +48,13 @@ dit_status dit_sched_allocate(const int32_t *gpus, const double *step_time, int3
  * q = min(s_i^m, floor(tau / T_i(A_i^m))) steps; options with q = 0 or A_i^m > n_gpus are dropped;
  * a request survives option o (or "none") iff t_now + tau + (remaining steps after o) * T_i^min <= D_i;
  * a group-knapsack DP over capacities 0..n_gpus maximises the number of survivors with at most one
- * option per request.  Outputs (each may be NULL except chosen): chosen[i] = option index or -1 for
- * "none", steps_done[i] = q of the choice (0 for none), the number of survivors and the GPUs used.
- * Among optimal plans the one found by scanning requests in order, capacities upward and options in
- * order (none first), keeping the first maximum, is returned.  O(R * N * options) time. */
+ * option per request.  Among plans with that many survivors the one that completes the most steps in
+ * the round is taken (the paper reaches a work-conserving plan through a separate scale-up pass over
+ * idle GPUs; here the DP's value is the pair (survivors, steps) compared in that order, so GPUs are
+ * not left idle while a request could use them).  Remaining ties: the plan found by scanning requests
+ * in order, capacities upward and options in order (none first), keeping the first maximum.
+ * Outputs (each may be NULL except chosen): chosen[i] = option index or -1 for "none", steps_done[i] =
+ * q of the choice (0 for none), the number of survivors and the GPUs used.  O(R * N * options) time. */
 dit_status dit_sched_round(const dit_sched_request *reqs, int32_t n_requests, int32_t n_gpus, double tau, double t_now,
                            int32_t *chosen, int32_t *steps_done, int32_t *n_survivors, int32_t *gpus_used);
 

@@ -52,6 +52,15 @@ def round_best(reqs, n_gpus: int, tau: float, t_now: float):
     return best, plans
 
 
+def round_best_progress(reqs, n_gpus: int, tau: float, t_now: float):
+    """Among the plans with the most survivors, those that complete the most steps in the round.
+    Returns (survivors, steps, plans)."""
+    best, plans = round_best(reqs, n_gpus, tau, t_now)
+    steps = [sum(option_progress(reqs[i][0][m], tau) for i, m in enumerate(p) if m >= 0) for p in plans]
+    top = max(steps) if steps else 0
+    return best, top, [p for p, s in zip(plans, steps) if s == top]
+
+
 def allocate_best(gpus: Sequence[int], step_time: Sequence[float], steps: int, budget: float):
     """Cheapest split over at most two degrees: returns (gpu_time, completion_time) or None if infeasible."""
     best = None

@@ -58,7 +58,6 @@ extern "C" dit_status dit_sched_round(const dit_sched_request* reqs, int32_t n_r
   }
   const double t_next = t_now + tau;
   const int N = n_gpus;
-  const int kNegInf = std::numeric_limits<int>::min() / 2;
   // per request: candidate options (index -1 = none), their width, progress and survival flag
   struct Cand { int option, width, q, survives; };
   std::vector<std::vector<Cand>> cands(n_requests);
@@ -76,17 +75,20 @@ extern "C" dit_status dit_sched_round(const dit_sched_request* reqs, int32_t n_r
       cands[i].push_back(Cand{m, o.gpus, q, survives(total - q)});
     }
   }
-  // dp[c]: most survivors among the requests processed so far with exactly c GPUs in use
-  std::vector<int> dp(N + 1, kNegInf), next(N + 1);
+  // dp[c]: best (survivors, steps completed this round), compared in that order, among the requests
+  // processed so far with exactly c GPUs in use; packed as survivors * 2^32 + steps
+  const long long kNegInf = std::numeric_limits<long long>::min() / 2;
+  std::vector<long long> dp(N + 1, kNegInf), next(N + 1);
   dp[0] = 0;
   std::vector<std::vector<int>> pick(n_requests, std::vector<int>(N + 1, -1));   // back-pointers: candidate index
   for (int i = 0; i < n_requests; ++i) {
     for (int c = 0; c <= N; ++c) {
-      int best = kNegInf, arg = -1;
+      long long best = kNegInf;
+      int arg = -1;
       for (size_t k = 0; k < cands[i].size(); ++k) {
         const Cand& o = cands[i][k];
         if (o.width > c || dp[c - o.width] == kNegInf) continue;
-        const int v = dp[c - o.width] + o.survives;
+        const long long v = dp[c - o.width] + (static_cast<long long>(o.survives) << 32) + o.q;
         if (v > best) { best = v; arg = static_cast<int>(k); }
       }
       next[c] = best;
@@ -97,7 +99,7 @@ extern "C" dit_status dit_sched_round(const dit_sched_request* reqs, int32_t n_r
   int c_star = 0;
   for (int c = 1; c <= N; ++c)
     if (dp[c] > dp[c_star]) c_star = c;
-  if (n_survivors) *n_survivors = dp[c_star] == kNegInf ? 0 : dp[c_star];
+  if (n_survivors) *n_survivors = dp[c_star] == kNegInf ? 0 : static_cast<int32_t>(dp[c_star] >> 32);
   if (gpus_used) *gpus_used = c_star;
   int c = c_star;
   for (int i = n_requests - 1; i >= 0; --i) {

@@ -79,8 +79,9 @@ def test_round_dp_matches_exhaustive_search():
         reqs = _random_instance(rng, int(rng.integers(0, 7)), n_gpus)
         tau, t_now = float(rng.choice([0.25, 0.5, 1.0])), float(rng.uniform(0, 3))
         chosen, done, surv, used = B.dit_sched_round(reqs, n_gpus, tau, t_now)
-        best, plans = S.round_best(reqs, n_gpus, tau, t_now)
+        best, steps, plans = S.round_best_progress(reqs, n_gpus, tau, t_now)
         assert surv == best, (trial, reqs, n_gpus, tau, t_now)
+        assert sum(done) == steps                          # and, among those, the most steps this round
         assert tuple(chosen) in plans                      # a valid optimal plan (several may exist)
         assert used == sum(reqs[i][0][m][1] for i, m in enumerate(chosen) if m >= 0) <= n_gpus
         for i, m in enumerate(chosen):
