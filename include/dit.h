@@ -306,7 +306,22 @@ dit_status dit_denoise_step(dit_ctx *ctx, float *latents, const void *text_token
                             int32_t n, const float *dsigma, const float *pooled, int32_t n_blocks,
                             float *velocity, void *stream);
 
-/* Number of kernel launches issued by the last dit_step_forward or dit_denoise_step on this context. */
+/* One scheduling round on this worker, as the paper's execution model has it (Section 5.2: in a
+ * round request i runs q_i consecutive steps; Section 5.3: requests of a batch leave it as they finish
+ * their steps): request r runs steps_in_round[r] >= 0 steps, all requests that still have a step left
+ * forming the packed batch of each step, so the batch shrinks as requests complete their quota.
+ *   sigmas  HOST [n, sigma_stride] fp32: sigmas[r, k] is request r's noise level before its k-th step
+ *           of this round and sigmas[r, k + 1] after it (sigma_stride >= largest step count + 1); the
+ *           step's diffusion time is t = 1000 * sigma, its Euler increment sigma[k + 1] - sigma[k]
+ *   latents, text_tokens, pooled: as for dit_denoise_step, for the FULL request list; latents are
+ *           updated in place, those of a request with no step left stay untouched
+ * Equal to calling dit_denoise_step once per step on the requests still active.  Asynchronous on
+ * `stream`; a few small device-to-device copies (pooled rows) are issued when the batch shrinks. */
+dit_status dit_denoise_round(dit_ctx *ctx, float *latents, const void *text_tokens, const dit_request *requests,
+                             int32_t n, const int32_t *steps_in_round, const float *sigmas, int32_t sigma_stride,
+                             const float *pooled, int32_t n_blocks, void *stream);
+
+/* Number of kernel launches issued by the last dit_step_forward, dit_denoise_step or dit_denoise_round on this context. */
 int64_t dit_last_launch_count(const dit_ctx *ctx);
 
 const char *dit_status_string(dit_status s);

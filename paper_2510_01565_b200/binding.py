@@ -28,7 +28,7 @@ EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
            "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
-           "dit_denoise_step", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
+           "dit_denoise_step", "dit_denoise_round", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
 
 class DitConfig(C.Structure):
@@ -136,6 +136,8 @@ def load_library() -> C.CDLL:
     lib.dit_sampler_update.argtypes = [vp, vp, vp, rq, i32, fp, vp]
     lib.dit_denoise_step.restype = C.c_int
     lib.dit_denoise_step.argtypes = [vp, vp, vp, rq, i32, fp, vp, i32, vp, vp]
+    lib.dit_denoise_round.restype = C.c_int
+    lib.dit_denoise_round.argtypes = [vp, vp, vp, rq, i32, C.POINTER(i32), fp, i32, vp, i32, vp]
     lib.dit_sched_allocate.restype = C.c_int
     lib.dit_sched_allocate.argtypes = [C.POINTER(i32), C.POINTER(C.c_double), i32, i32, C.c_double,
                                        C.POINTER(DitSchedOption), C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i32)]
@@ -451,6 +453,21 @@ class DitContext:
         self._check(self.lib.dit_denoise_step(self.handle, self._ptr(latents), self._ptr(text_tokens), request_array(reqs), n,
                                               ds.ctypes.data_as(C.POINTER(C.c_float)), self._ptr(pooled), n_blocks,
                                               self._ptr(velocity), self._stream(stream)))
+        return latents
+
+    def dit_denoise_round(self, latents, text_tokens, reqs, steps_in_round, sigmas, pooled, n_blocks: int, stream=None):
+        """steps_in_round: [n] ints; sigmas: [n, max_steps + 1] floats (host).  Latents updated in place."""
+        n = len(reqs)
+        steps = np.ascontiguousarray(np.asarray(steps_in_round, dtype=np.int32))
+        sig = np.ascontiguousarray(np.asarray(sigmas, dtype=np.float32))
+        assert steps.shape == (n,) and sig.ndim == 2 and sig.shape[0] == n
+        self._f32(latents)
+        if pooled is not None:
+            self._f32(pooled, n * self.cond_dim)
+        self._check(self.lib.dit_denoise_round(self.handle, self._ptr(latents), self._ptr(text_tokens), request_array(reqs), n,
+                                               steps.ctypes.data_as(C.POINTER(C.c_int32)),
+                                               sig.ctypes.data_as(C.POINTER(C.c_float)), sig.shape[1], self._ptr(pooled),
+                                               n_blocks, self._stream(stream)))
         return latents
 
     def dit_ctx_poll_status(self):

@@ -38,7 +38,7 @@ struct Layout {
   size_t weights, stream, h, qkv, a, u, mod, status, stage_tokens, stage_cond, stage_out;
   // tensors and intermediates of the shell around the block stack
   size_t sh_w_in, sh_b_in, sh_w_t1, sh_b_t1, sh_w_t2, sh_b_t2, sh_w_fa, sh_b_fa, sh_w_out, sh_b_out;
-  size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok;
+  size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok, sh_pooled;
   size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
   size_t row_scale;    // per-row scales of the e4m3 activations (DIT_FLAG_FP8_GEMM)
   size_t items;        // two-stream launches: [0] item count, then per-tile flags, then the items
@@ -108,6 +108,7 @@ Layout make_layout(const dit_config& c) {
   L.sh_cond = take(R * C * 2);
   L.sh_modfin = take(R * 2 * H * 4);
   L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
+  L.sh_pooled = take(R * C * 4);
   L.rope_theta = take(64 * 4);
   L.row_scale = take(T * 4);
   L.items = take((16 + 3 * (T / (2 * 128) + 2)) * 4);
@@ -879,11 +880,13 @@ const char* dit_last_error(const dit_ctx* ctx) { return ctx ? ctx->err : ""; }
 namespace {
 
 // Packed-batch and per-request geometry from a HOST request array (same rules as dit_pack_requests).
-dit_status build_shell(dit_ctx* ctx, const dit_request* reqs, int n, const float* dsigma, SeqInfo* seq, ShellInfo* info) {
+dit_status build_shell(dit_ctx* ctx, const dit_request* reqs, int n, const float* dsigma, SeqInfo* seq, ShellInfo* info,
+                       int* total_text = nullptr) {
   if (n > ctx->cfg.max_requests) return fail(ctx, DIT_ERR_CAPACITY, "n exceeds max_requests");
   int32_t lens[DIT_MAX_REQUESTS];
   long long total = 0;
-  info->img_cu[0] = 0; info->txt_cu[0] = 0;
+  info->img_cu[0] = 0;
+  int txt_rows = 0;
   for (int r = 0; r < n; ++r) {
     const dit_request& q = reqs[r];
     if (q.height <= 0 || q.width <= 0 || q.height % 16 || q.width % 16 || q.n_text_tokens < 0)
@@ -892,13 +895,16 @@ dit_status build_shell(dit_ctx* ctx, const dit_request* reqs, int n, const float
     total += n_img + q.n_text_tokens;
     if (total > ctx->cfg.max_total_tokens) return fail(ctx, DIT_ERR_CAPACITY, "packed batch exceeds max_total_tokens");
     lens[r] = static_cast<int32_t>(n_img + q.n_text_tokens);
+    info->lat_off[r] = 64ll * info->img_cu[r];
+    info->txt_row[r] = txt_rows;
     info->img_cu[r + 1] = info->img_cu[r] + static_cast<int>(n_img);
-    info->txt_cu[r + 1] = info->txt_cu[r] + q.n_text_tokens;
+    txt_rows += q.n_text_tokens;
     info->gw[r] = q.width / 16;
     info->t[r] = q.timestep;
     info->dsigma[r] = dsigma ? dsigma[r] : 0.f;
   }
   if (!build_seq(lens, n, seq)) return fail(ctx, DIT_ERR_INTERNAL, "empty request");
+  if (total_text) *total_text = txt_rows;
   return DIT_OK;
 }
 
@@ -1042,9 +1048,10 @@ dit_status dit_embed_latents(dit_ctx* ctx, const float* latents, const void* tex
   if (s != DIT_OK || n == 0) return s;
   if (!latents || !packed_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
   SeqInfo seq{}; ShellInfo info{};
-  s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
+  int total_text = 0;
+  s = build_shell(ctx, reqs, n, nullptr, &seq, &info, &total_text);
   if (s != DIT_OK) return s;
-  if (info.txt_cu[n] > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
+  if (total_text > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
   return embed_impl(ctx, latents, text_tokens, seq, info, packed_tokens, static_cast<cudaStream_t>(stream));
 }
 
@@ -1104,9 +1111,10 @@ dit_status dit_denoise_step(dit_ctx* ctx, float* latents, const void* text_token
   for (int b = 0; b < n_blocks; ++b)
     if (!ctx->blocks[b].loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "a block in [0, n_blocks) has no weights");
   SeqInfo seq{}; ShellInfo info{};
-  s = build_shell(ctx, reqs, n, dsigma, &seq, &info);
+  int total_text = 0;
+  s = build_shell(ctx, reqs, n, dsigma, &seq, &info, &total_text);
   if (s != DIT_OK) return s;
-  if (info.txt_cu[n] > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
+  if (total_text > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* cond = ctx->ws + ctx->lay.sh_cond;
   void* tokens = ctx->ws + ctx->lay.stage_tokens;
@@ -1123,6 +1131,77 @@ dit_status dit_denoise_step(dit_ctx* ctx, float* latents, const void* text_token
   s = final_impl(ctx, x, seq, info, n, cond, velocity, latents, st);
   if (s != DIT_OK) return s;
   ctx->last_launches += 3 + 1 + 4;
+  return DIT_OK;
+}
+
+dit_status dit_denoise_round(dit_ctx* ctx, float* latents, const void* text_tokens, const dit_request* reqs, int32_t n,
+                             const int32_t* steps_in_round, const float* sigmas, int32_t sigma_stride, const float* pooled,
+                             int32_t n_blocks, void* stream) {
+  dit_status s = check_shell_args(ctx, reqs, n);
+  if (s != DIT_OK || n == 0) return s;
+  if (!latents || !steps_in_round || !sigmas) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  if (n_blocks < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "n_blocks must be at least 1");
+  if (n_blocks > ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "n_blocks exceeds max_blocks");
+  for (int b = 0; b < n_blocks; ++b)
+    if (!ctx->blocks[b].loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "a block in [0, n_blocks) has no weights");
+  int max_steps = 0;
+  for (int r = 0; r < n; ++r) {
+    if (steps_in_round[r] < 0) return fail(ctx, DIT_ERR_INVALID_ARG, "negative step count");
+    max_steps = std::max(max_steps, steps_in_round[r]);
+  }
+  if (sigma_stride < max_steps + 1) return fail(ctx, DIT_ERR_INVALID_ARG, "sigma_stride must be at least the largest step count + 1");
+  SeqInfo full_seq{}; ShellInfo full{};
+  int total_text = 0;
+  s = build_shell(ctx, reqs, n, nullptr, &full_seq, &full, &total_text);     // also checks shapes and capacity
+  if (s != DIT_OK) return s;
+  if (total_text > 0 && !text_tokens) return fail(ctx, DIT_ERR_INVALID_ARG, "text_tokens is NULL but a request has text tokens");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t Cd = ctx->cfg.cond_dim;
+  void* cond = ctx->ws + ctx->lay.sh_cond;
+  void* tokens = ctx->ws + ctx->lay.stage_tokens;
+  float* x = ctx->at<float>(ctx->lay.stream);
+  float* pooled_stage = ctx->at<float>(ctx->lay.sh_pooled);
+  int64_t launches = 0;
+  for (int k = 0; k < max_steps; ++k) {
+    // the requests that still have a step to run in this round, in their original order
+    SeqInfo seq{}; ShellInfo info{};
+    int32_t lens[DIT_MAX_REQUESTS];
+    int active[DIT_MAX_REQUESTS];
+    int na = 0;
+    info.img_cu[0] = 0;
+    for (int r = 0; r < n; ++r) {
+      if (steps_in_round[r] <= k) continue;
+      const int n_img = full.img_cu[r + 1] - full.img_cu[r];
+      lens[na] = full_seq.cu[r + 1] - full_seq.cu[r];
+      info.img_cu[na + 1] = info.img_cu[na] + n_img;
+      info.lat_off[na] = full.lat_off[r];
+      info.txt_row[na] = full.txt_row[r];
+      info.gw[na] = full.gw[r];
+      const float s0 = sigmas[static_cast<size_t>(r) * sigma_stride + k], s1 = sigmas[static_cast<size_t>(r) * sigma_stride + k + 1];
+      info.t[na] = 1000.0f * s0;
+      info.dsigma[na] = s1 - s0;
+      active[na] = r;
+      ++na;
+    }
+    if (!build_seq(lens, na, &seq)) return fail(ctx, DIT_ERR_INTERNAL, "empty request");
+    const float* pooled_k = pooled;
+    if (pooled && na != n) {   // the batch has shrunk: line the active requests' pooled rows up
+      for (int i = 0; i < na; ++i)
+        DIT_CUDA_TRY(ctx, cudaMemcpyAsync(pooled_stage + i * Cd, pooled + active[i] * Cd, Cd * 4, cudaMemcpyDeviceToDevice, st));
+      pooled_k = pooled_stage;
+    }
+    s = cond_impl(ctx, info, na, pooled_k, cond, st);
+    if (s != DIT_OK) return s;
+    s = embed_impl(ctx, latents, text_tokens, seq, info, tokens, st);
+    if (s != DIT_OK) return s;
+    const RowGeom geo = geom_of(info);
+    s = step_impl(ctx, tokens, lens, na, cond, n_blocks, x, st, &geo);
+    if (s != DIT_OK) return s;
+    s = final_impl(ctx, x, seq, info, na, cond, nullptr, latents, st);
+    if (s != DIT_OK) return s;
+    launches += ctx->last_launches + 3 + 1 + 4;
+  }
+  ctx->last_launches = launches;
   return DIT_OK;
 }
 

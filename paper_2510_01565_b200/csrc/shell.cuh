@@ -12,8 +12,10 @@ constexpr int kTEmbDim = DIT_T_EMB_DIM;
 
 // Per-request geometry of a step, passed by value as a kernel parameter.
 struct ShellInfo {
-  int img_cu[DIT_MAX_REQUESTS + 1];   // prefix sums of image tokens: request r's latent starts at 64 * img_cu[r] floats
-  int txt_cu[DIT_MAX_REQUESTS + 1];   // prefix sums of text tokens: rows of the text buffer
+  int img_cu[DIT_MAX_REQUESTS + 1];   // prefix sums of image tokens over the requests of this launch
+  long long lat_off[DIT_MAX_REQUESTS];// first float of request r's latent in the latent buffer (64 * its image-token prefix
+                                      // in the caller's full request list, which may be longer than this launch's)
+  int txt_row[DIT_MAX_REQUESTS];      // first row of request r's text tokens in the text buffer
   int gw[DIT_MAX_REQUESTS];           // patch columns (width / 16)
   float t[DIT_MAX_REQUESTS];          // diffusion time of this step
   float dsigma[DIT_MAX_REQUESTS];     // sigma_next - sigma_cur
@@ -35,7 +37,7 @@ timestep_embed_kernel(const __grid_constant__ ShellInfo info, float* __restrict_
 // ------------------------------------------------------------------------------------------------
 // Patch embedding + 2-D sine/cosine position + text rows -> packed bf16 tokens.
 //   image row (py, px) of request r:  tok = patch(py, px) W_in + b_in + pos(py, px)
-//   text row i of request r:          tok = text[txt_cu[r] + i]
+//   text row i of request r:          tok = text[txt_row[r] + i]
 // A CTA covers 64 packed rows x 128 channels: the 64 patches (fp32) and the 64 x 128 slice of W_in
 // (bf16) sit in shared memory; a thread owns 4 rows x 8 channels.  The latent is read as float2
 // (the two dx of a patch row), consecutive threads taking consecutive patches of a grid row.
@@ -61,7 +63,7 @@ embed_latents_kernel(const float* __restrict__ latents, const __nv_bfloat16* __r
       const int local = row - seq.cu[req];
       const int n_img = info.img_cu[req + 1] - info.img_cu[req];
       if (local < n_img) { py = local / info.gw[req]; px = local - py * info.gw[req]; }
-      else { py = -1; px = info.txt_cu[req] + (local - n_img); }
+      else { py = -1; px = info.txt_row[req] + (local - n_img); }
     }
     s_req[tid] = req; s_py[tid] = py; s_px[tid] = px;
   }
@@ -80,7 +82,7 @@ embed_latents_kernel(const float* __restrict__ latents, const __nv_bfloat16* __r
       const int gw = info.gw[req], w8 = 2 * gw;
       const long long plane = 4ll * (info.img_cu[req + 1] - info.img_cu[req]);
       const int c = pair >> 1, dy = pair & 1;
-      const float* src = latents + 64ll * info.img_cu[req] + c * plane + static_cast<long long>(2 * py + dy) * w8 + 2 * s_px[r];
+      const float* src = latents + info.lat_off[req] + c * plane + static_cast<long long>(2 * py + dy) * w8 + 2 * s_px[r];
       v = __ldg(reinterpret_cast<const float2*>(src));
     }
     s_patch[r][2 * pair] = v.x;
@@ -165,7 +167,7 @@ unpatchify_update_kernel(const float* __restrict__ v_tok, float* __restrict__ ve
     const int gw = info.gw[req], w8 = 2 * gw;
     const int py = local / gw, px = local - py * gw;
     const int c = pair >> 1, dy = pair & 1;
-    const long long off = 64ll * info.img_cu[req] + c * (4ll * n_img) + static_cast<long long>(2 * py + dy) * w8 + 2 * px;
+    const long long off = info.lat_off[req] + c * (4ll * n_img) + static_cast<long long>(2 * py + dy) * w8 + 2 * px;
     const float2 v = *reinterpret_cast<const float2*>(v_tok + static_cast<size_t>(row) * kPatchDim + 2 * pair);
     if (velocity) *reinterpret_cast<float2*>(velocity + off) = v;
     if (latents) {

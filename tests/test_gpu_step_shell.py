@@ -249,3 +249,53 @@ def test_shell_argument_errors(B):
     torch.cuda.synchronize()
     ctx.dit_ctx_poll_status()
     ctx.close()
+
+
+def test_round_with_uneven_step_counts(B):
+    # one scheduling round on a worker: each request runs its own number of steps, the packed batch
+    # shrinks as requests use up their quota (the second request runs no step at all)
+    import torch
+    reqs = [(64, 96, 5), (32, 32, 0), (96, 32, 2), (32, 64, 7)]
+    si = W.make_step_inputs(W.SMALL, 2, reqs, seed=19)
+    run = ShellRun(B, si, 2)
+    steps = [3, 0, 1, 2]
+    sig = np.zeros((4, 4), dtype=np.float32)
+    for r, start in enumerate([1.0, 0.5, 0.62, 0.3]):
+        sig[r] = np.float32(start) - np.float32(0.07) * np.arange(4, dtype=np.float32) * np.float32(1 + 0.1 * r)
+    before = run.latents.clone()
+    run.ctx.dit_denoise_round(run.latents, run.text, si.requests, steps, sig, run.pooled, 2)
+    run.sync()
+    assert run.ctx.dit_last_launch_count() == 3 * ((1 + 7 * 2) + 8)
+    shell, blocks = f64w(si.shell), [f64w(w) for w in si.weights[:2]]
+    for r in range(4):
+        z = si.latents[r].astype(np.float64)
+        for k in range(steps[r]):
+            t = float(np.float32(1000.0) * sig[r, k])
+            ds = float(sig[r, k + 1] - sig[r, k])
+            (z,), _, _ = S.denoise_step([z], [W.bf16_to_f64(si.texts[r])], [t], [ds], [si.pooled[r].astype(np.float64)],
+                                        shell, blocks, si.dims.n_heads, si.dims.ln_eps)
+        got = run.latent_of(run.latents, r)
+        if steps[r] == 0:
+            assert np.array_equal(got, si.latents[r].astype(np.float64))       # untouched
+        else:
+            err = O.error_metric(got - si.latents[r].astype(np.float64), z - si.latents[r].astype(np.float64))
+            assert err <= TOL, f"request {r} after {steps[r]} steps: {err:.3e}"
+    # the same round as separate steps on the shrinking request lists, bit for bit
+    z2 = before.clone()
+    for k in range(3):
+        act = [r for r in range(4) if steps[r] > k]
+        qs = [W.Request(si.requests[r].height, si.requests[r].width, si.requests[r].n_text_tokens,
+                        float(np.float32(1000.0) * sig[r, k]), 0) for r in act]
+        lat = torch.cat([z2[int(run.lat_cu[r]):int(run.lat_cu[r + 1])] for r in act])
+        txt = [B.bits_to_cuda_bf16(si.texts[r]) for r in act if si.texts[r].shape[0]]
+        txt = torch.cat(txt) if txt else None
+        ds = np.array([sig[r, k + 1] - sig[r, k] for r in act], dtype=np.float32)
+        run.ctx.dit_denoise_step(lat, txt, qs, ds, run.pooled[act].contiguous(), 2)
+        p = 0
+        for r in act:
+            m = int(run.lat_cu[r + 1] - run.lat_cu[r])
+            z2[int(run.lat_cu[r]):int(run.lat_cu[r + 1])] = lat[p:p + m]
+            p += m
+    run.sync()
+    assert torch.equal(z2, run.latents)
+    run.close()
