@@ -227,7 +227,8 @@ dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *laun
  * and nothing else).  It needs no context and no workspace.
  *   mod_out[r, :] = W_ada^T SiLU(cond[r, :]) + b_ada        device [n_requests, 6H] fp32
  *   cond device [n_requests, C] bf16; w_ada device [C, 6H] bf16; b_ada device [6H] bf16 or NULL (zero)
- * The result equals the `mod` vectors dit_step_forward computes for that block.  The fp32 copy of
+ * The result is that of the `mod` vectors dit_step_forward computes for that block (the same kernel; a
+ * context with many blocks may sum the cond channels in wider groups, which moves the last fp32 bits).  The fp32 copy of
  * the bias, which the context path keeps in the caller's workspace, lives here in a fixed 96 KiB
  * array inside the library image (every GPU that loads the library holds it until the process
  * exits).  Limits: hidden a multiple of 64 and <= 4096, cond_dim <= 4096, n_requests <=

@@ -8,16 +8,18 @@ namespace dit {
 // ------------------------------------------------------------------------------------------------
 // adaLN modulation for all blocks at once:
 //   mod[r, b, j] = sum_c SiLU(cond[r, c]) * W_ada_b[c, j] + b_ada_b[j],   j in [0, 6H)
-// Bound by reading W_ada once (C x 6H bf16 per block).  A CTA owns 128 consecutive columns of one
-// block: 16 column groups (8 bf16 = 16 B per load) x 16 slices of the C range; slice partials are
-// combined in shared memory in slice order, so the result does not depend on the number of requests.
+// Bound by reading W_ada once (C x 6H bf16 per block).  A CTA owns kModCols consecutive columns of one
+// block: kModCols / 8 column groups (8 bf16 = 16 B per load) x 256 / (kModCols / 8) slices of the C range;
+// slice partials are combined in shared memory in slice order, so the result does not depend on the
+// number of requests.  The strip width is chosen per launch: the widest that still gives every SM about two
+// CTAs (wide strips read 1-2 KB runs of a row instead of 256 B, which DRAM serves much better).
 // The partials reuse the activation buffer, which keeps two CTAs resident per SM.
 // Requests are processed in groups of kModReqGroup to bound registers.
 // ------------------------------------------------------------------------------------------------
 constexpr int kModReqGroup = 8;
 constexpr int kModThreads = 256;
-constexpr int kModCols = 128;
-constexpr int kModSlices = 16;
+constexpr int kModColsMin = 128;   // narrowest strip of columns a CTA owns; wider strips (template argument) read longer
+                                   // contiguous runs of each W_ada row and are used when there are CTAs to spare
 constexpr int kModBatch = 12;
 
 struct ModParams {
@@ -37,13 +39,14 @@ struct ModParams {
 // 2 = fp32 in32 as it is.
 enum ModInput : int { kModInCondSilu = 0, kModInF32Silu = 1, kModInF32 = 2 };
 
-template <int kIn>
+template <int kIn, int kModCols = kModColsMin>
 __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams p) {
+  constexpr int kModSlices = kModThreads / (kModCols / 8);
   extern __shared__ float sm[];                       // silu(cond) [G][C]; afterwards reused for partials [16][G][128]
   const int cols_per_block = (p.N6 + kModCols - 1) / kModCols;
   const int blk = blockIdx.x / cols_per_block;
   const int col_base = (blockIdx.x % cols_per_block) * kModCols;
-  const int cg = threadIdx.x & 15, slice = threadIdx.x >> 4;
+  const int cg = threadIdx.x % (kModCols / 8), slice = threadIdx.x / (kModCols / 8);
   const int col = col_base + cg * 8;
   const __nv_bfloat16* w = p.w_ada0 + blk * p.w_block_stride;
   const float* bias = p.b_ada0 + blk * p.b_block_stride;
