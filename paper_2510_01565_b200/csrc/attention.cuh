@@ -10,16 +10,20 @@
 // row maximum is taken.
 //
 // Per KV tile j (128 keys) and query tile i (online softmax, fp32 statistics):
-//   MMA warp      S_i = Q_i K_j^T              -> TMEM S[i]            (SS tcgen05.mma)
-//   softmax WG i  m, alpha, P = exp2(c*(S-m))  -> fp16 P over S[i]'s columns (tcgen05.st)
+//   MMA warp      S_i = Q_i K_j^T              -> TMEM S (one buffer, used by the two tiles in turn)
+//   softmax WG i  reads S into registers and hands the buffer back at once;
+//                 m, alpha, P = exp2(c*(S-m))  -> fp16 P[i] in its own TMEM columns (tcgen05.st)
 //   MMA warp      O_i += P_i V_j               -> TMEM O[i]            (TS tcgen05.mma, A = P in TMEM)
+// Because P does not overwrite S, the scores of a tile's NEXT key block are computed while its
+// softmax warpgroup is still busy with the current one: S uses run one and a half key blocks ahead
+// of the P V products (order on the tensor pipe: P V of tile 0, scores of tile 1, P V of tile 1,
+// scores of tile 0, ...), so a warpgroup finds its next scores waiting instead of standing idle for a
+// P V + Q K^T round trip.  TMEM: S 128 columns, P[0], P[1] 64 each, O[0], O[1] 128 each = 512.
 // O is rescaled in TMEM only when a row maximum has grown by more than 2^8 since the reference was
 // set (rare after the first tiles); P is bounded by 2^8, and O and l share the reference, so the
-// normalised result is the same.
-// The two warpgroups alternate: while one exponentiates, the tensor core runs the other's P V and
-// next Q K^T.  Output = acc / l, written as fp16 [T, H].
+// normalised result is the same.  Output = acc / l, written as fp16 [T, H].
 //
-// Thread layout (384): warpgroup 0 = {warp 0: TMA producer, warp 1: MMA issuer + TMEM owner},
+// Thread layout (384): warpgroup 0 = {warp 0: TMA producer, warp 1: score MMAs + TMEM owner, warp 2: P V MMAs},
 // warpgroups 1 and 2 = softmax for query tile 0 and 1.  Registers are re-balanced with setmaxnreg.
 #pragma once
 #include "common.cuh"
@@ -76,7 +80,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   auto s_full = [&](int i) { return bar0 + 8u * (9 + i); };
   auto p_full = [&](int i) { return bar0 + 8u * (11 + i); };
   auto o_full = [&](int i) { return bar0 + 8u * (13 + i); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + C::OFF_BAR + 8 * 15);
+  const uint32_t s_free = bar0 + 8u * 15;      // the warpgroup that was handed S has read it into registers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + C::OFF_BAR + 8 * 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -99,6 +104,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
+    mbar_init(s_free, 128);
     for (int s = 0; s < 2; ++s) {
       mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1);
       mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1);
@@ -113,9 +119,9 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // TMEM columns: S[0] 0..127, S[1] 128..255 (P[i] overwrites the first 64 columns of S[i]),
+  // TMEM columns: S 0..127 (shared by the two query tiles in turn), P[0] 128..191, P[1] 192..255,
   // O[0] 256.., O[1] 384..
-  const uint32_t tS = tmem_base, tO = tmem_base + 256;
+  const uint32_t tS = tmem_base, tP = tmem_base + 128, tO = tmem_base + 256;
 
   if (warp < 4) {
     DIT_SETMAXNREG_DEC(96);
@@ -139,50 +145,54 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
           tma_load_2d(base + C::OFF_V + s * C::TILE_BYTES + pn * C::PANEL, &tmQKV, xv + pn * 64, y, v_full(s));
       }
     } else if (warp == 1 && lane == 0) {
-      // ------------------------------------------------------------------ MMA issuer
+      // ------------------------------------------------------------------ MMA issuer 1: scores
+      // Uses of the S buffer run in the order (j, i) = (0,0), (0,1), (1,0), ...; use u = j * ntile + i.
+      // A use waits for its K tile (first query tile) and for the warpgroup of use u - 1 to have read
+      // the buffer out; the K stage is released after the last query tile.  This thread and the P V
+      // issuer wait independently, so neither hand-off keeps the other's MMAs off the tensor pipe.
       constexpr uint32_t idesc_s = idesc_f16(128, 128, false);
-      constexpr uint32_t idesc_pv = idesc_f16(128, D, true);
       const int ntile = tile1_valid ? 2 : 1;
-      // Descriptors are built once; inside the loops only constant offsets are added (>> 4 units).
       static_assert(C::KV_STAGES == 2, "descriptor selection below assumes two stages");
       const uint64_t qdesc0 = smem_desc_sw128(base + C::OFF_Q, 16, 1024);
       const uint64_t kdesc0 = smem_desc_sw128(base + C::OFF_K, 16, 1024);
-      // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns live
-      // one panel further (leading byte offset).
-      const uint64_t vdesc0 = smem_desc_sw128(base + C::OFF_V, C::PANEL, 1024);
       constexpr uint32_t kTileStep = C::TILE_BYTES >> 4;
-      // S_i(j) = Q_i K_j^T; the K stage is released after the last query tile has used it
-      auto issue_s = [&](int j, int i) {
+      if (!mbar_wait(q_full, 0, abort_flag)) goto done;
+      const int total = ntile * nkv;
+      for (int u = 0, j = 0, i = 0; u < total; ++u) {
         const int s = j % C::KV_STAGES;
+        if (i == 0 && !mbar_wait(k_full(s), (j / C::KV_STAGES) & 1u, abort_flag)) goto done;
+        if (u > 0 && !mbar_wait(s_free, (u - 1) & 1u, abort_flag)) goto done;
+        tc_fence_after();
         const uint64_t qd = qdesc0 + i * kTileStep, kd = kdesc0 + s * kTileStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = ((kk >> 2) * C::PANEL + (kk & 3) * 32) >> 4;
-          umma_f16(tS + i * 128, qd + off, kd + off, idesc_s, kk != 0);
+          umma_f16(tS, qd + off, kd + off, idesc_s, kk != 0);
         }
         if (i == ntile - 1) umma_commit(k_empty(s));
         umma_commit(s_full(i));
-      };
-      if (!mbar_wait(q_full, 0, abort_flag)) goto done;
-      if (!mbar_wait(k_full(0), 0, abort_flag)) goto done;
-      tc_fence_after();
-      for (int i = 0; i < ntile; ++i) issue_s(0, i);
+        if (++i == ntile) { i = 0; ++j; }
+      }
+    } else if (warp == 2 && lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer 2: P V
+      constexpr uint32_t idesc_pv = idesc_f16(128, D, true);
+      const int ntile = tile1_valid ? 2 : 1;
+      // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns live
+      // one panel further (leading byte offset).
+      const uint64_t vdesc0 = smem_desc_sw128(base + C::OFF_V, C::PANEL, 1024);
+      constexpr uint32_t kTileStep = C::TILE_BYTES >> 4;
       for (int j = 0; j < nkv; ++j) {
-        const int s = j % C::KV_STAGES; const uint32_t ph = (j / C::KV_STAGES) & 1u;
-        // operands of this round were requested a whole round ago: check them off the critical path
-        if (!mbar_wait(v_full(s), ph, abort_flag)) goto done;
-        if (j + 1 < nkv && !mbar_wait(k_full((j + 1) % C::KV_STAGES), ((j + 1) / C::KV_STAGES) & 1u, abort_flag)) goto done;
+        const int s = j % C::KV_STAGES;
+        if (!mbar_wait(v_full(s), (j / C::KV_STAGES) & 1u, abort_flag)) goto done;
+        const uint64_t vd = vdesc0 + s * kTileStep;
         for (int i = 0; i < ntile; ++i) {
           if (!mbar_wait(p_full(i), j & 1u, abort_flag)) goto done;
           tc_fence_after();
-          const uint64_t vd = vdesc0 + s * kTileStep;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)         // 16 keys per MMA: 8 TMEM columns of packed fp16 P
-            umma_f16_ts(tO + i * 128, tS + i * 128 + kk * 8, vd + kk * (2048 >> 4), idesc_pv, (j | kk) != 0);
+            umma_f16_ts(tO + i * 128, tP + i * 64 + kk * 8, vd + kk * (2048 >> 4), idesc_pv, (j | kk) != 0);
           if (i == ntile - 1) umma_commit(v_empty(s));
           umma_commit(o_full(i));
-          // the next scores of this tile go over P_i: the tensor pipe runs them after the P V above
-          if (j + 1 < nkv) issue_s(j + 1, i);
         }
       }
     }
@@ -194,7 +204,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
     const int prow = quarter * 32 + lane;                        // query row inside the tile
     if (len == 0 || (tile == 1 && !tile1_valid)) goto done;
     const uint32_t lane_sel = static_cast<uint32_t>(quarter * 32) << 16;
-    const uint32_t tSi = tS + tile * 128 + lane_sel, tOi = tO + tile * 128 + lane_sel;
+    const uint32_t tSi = tS + lane_sel, tPi = tP + tile * 64 + lane_sel, tOi = tO + tile * 128 + lane_sel;
     const float c = p.scale_log2;
     const float2 c2 = make_float2(c, c);
     // Running reference maximum m_ref (scores are exponentiated relative to it) and row sum l.
@@ -214,6 +224,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) tmem_ld32p(tSi + ch * 32, sv + ch * 32);
       tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(s_free);                                       // the scores are in registers: S may be overwritten
       if (valid < 128) {
 #pragma unroll
         for (int i = 0; i < 128; ++i)
@@ -233,7 +245,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       } else {
         const bool grow = (mx - m_ref) * c > kRescaleLog2;
         if (__any_sync(0xffffffffu, grow)) {
-          // rare: rescale this warp's rows of O (rows that did not grow are multiplied by 1)
+          // rare: rescale this warp's rows of O (rows that did not grow are multiplied by 1); the
+          // previous P V, which accumulates into O, must have finished
           if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), (j - 1) & 1u, abort_flag))) goto done;
           tc_fence_after();
           const float alpha = grow ? exp2_approx((m_ref - mx) * c) : 1.0f;
@@ -253,21 +266,25 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       }
       const float neg_mc = -m_ref * c;
       const float2 nm2 = make_float2(neg_mc, neg_mc);
-      // P = exp2(c*s - c*m_ref) as fp16 over the columns S occupied, row sum in fp32
+      // P = exp2(c*s - c*m_ref) as fp16, packed in place over the score registers (pair k lands in
+      // word k, which has been consumed by then); row sum in fp32
       float2 rs0 = make_float2(0.f, 0.f), rs1 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float2 x = ffma2(make_float2(__uint_as_float(sv[ch * 32 + i]), __uint_as_float(sv[ch * 32 + i + 1])), c2, nm2);
-          const float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
-          if (i & 2) rs1 = fadd2(rs1, e); else rs0 = fadd2(rs0, e);
-          const __half2 hh = __floats2half2_rn(e.x, e.y);
-          w[i >> 1] = *reinterpret_cast<const uint32_t*>(&hh);
-        }
-        tmem_st16(tSi + ch * 16, w);
+      for (int i = 0; i < 128; i += 2) {
+        const float2 x = ffma2(make_float2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2);
+        const float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
+        if (i & 2) rs1 = fadd2(rs1, e); else rs0 = fadd2(rs0, e);
+        const __half2 hh = __floats2half2_rn(e.x, e.y);
+        sv[i >> 1] = *reinterpret_cast<const uint32_t*>(&hh);
       }
+      // P[tile] is still being read by the previous key block's P V until that product has finished;
+      // by now (a whole tile of exponentials later) it normally has
+      if (j > 0) {
+        if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), (j - 1) & 1u, abort_flag))) goto done;
+        tc_fence_after();
+      }
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) tmem_st16(tPi + ch * 16, *reinterpret_cast<const uint32_t(*)[16]>(sv + ch * 16));
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(p_full(tile));
