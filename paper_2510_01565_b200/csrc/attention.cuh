@@ -104,11 +104,11 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    mbar_init(s_free, 128);
+    mbar_init(s_free, 4);                      // one arrival per warp of the warpgroup
     for (int s = 0; s < 2; ++s) {
       mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1);
       mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1);
-      mbar_init(s_full(s), 1); mbar_init(p_full(s), 128); mbar_init(o_full(s), 1);
+      mbar_init(s_full(s), 1); mbar_init(p_full(s), 4); mbar_init(o_full(s), 1);
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -225,7 +225,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       for (int ch = 0; ch < 4; ++ch) tmem_ld32p(tSi + ch * 32, sv + ch * 32);
       tmem_ld_wait();
       tc_fence_before();
-      mbar_arrive(s_free);                                       // the scores are in registers: S may be overwritten
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_free);                        // the scores are in registers: S may be overwritten
       if (valid < 128) {
 #pragma unroll
         for (int i = 0; i < 128; ++i)
@@ -287,7 +288,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       for (int ch = 0; ch < 4; ++ch) tmem_st16(tPi + ch * 16, *reinterpret_cast<const uint32_t(*)[16]>(sv + ch * 16));
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(p_full(tile));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full(tile));
       l += (rs0.x + rs0.y) + (rs1.x + rs1.y);
     }
     {
