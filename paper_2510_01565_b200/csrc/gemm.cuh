@@ -216,10 +216,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const float* gate = p.gate + ((DUAL && kind) ? p.gate_kind_stride : 0);
       const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
       const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
-      // Residual rows of this tile do not depend on the accumulator: the first two 32-column chunks
-      // are requested before waiting for the MMAs, later chunks two iterations ahead.
+      // Residual rows of this tile do not depend on the accumulator: the first four 32-column chunks
+      // are requested before waiting for the MMAs, later chunks four iterations ahead.
       const int cg = (lane & 7) * 4;
-      float4 xres[2][8];
+      constexpr int kResDepth = 4;             // 32-column chunks of residual rows in flight per lane
+      float4 xres[kResDepth][8];
       auto load_resid = [&](int c, float4 (&x)[8]) {
         const int col = n0 + c * 32 + cg;
         if (EPI == kEpiGateResidF32 && col < p.N) {
@@ -230,8 +231,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       };
-      load_resid(0, xres[0]);
-      load_resid(1, xres[1]);
+#pragma unroll
+      for (int d = 0; d < kResDepth; ++d) load_resid(d, xres[d]);
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
@@ -329,8 +330,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             float4 x[8];
             if (EPI == kEpiGateResidF32) {
 #pragma unroll
-              for (int it = 0; it < 8; ++it) x[it] = xres[c & 1][it];
-              if (c + 2 < BN / 32) load_resid(c + 2, xres[c & 1]);
+              for (int it = 0; it < 8; ++it) x[it] = xres[c % kResDepth][it];
+              if (c + kResDepth < BN / 32) load_resid(c + kResDepth, xres[c % kResDepth]);
             }
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
