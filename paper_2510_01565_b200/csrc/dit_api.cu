@@ -406,9 +406,6 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     AttnParams ap{};
     ap.out = bs.parallel ? cat : a; ap.ld_out = bs.parallel ? H + F : H;
     ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
-#ifdef DIT_ATTN_TRACE
-    { const char* e_ = getenv("DIT_TRACE_PTR"); ap.trace = e_ ? reinterpret_cast<long long*>(strtoull(e_, nullptr, 0)) : nullptr; }
-#endif
     ap.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c.head_dim));
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_ATTENTION, [&] {
       return c.head_dim == 128 ? launch_attention<128>(tm_qkv, ap, seq, st) : launch_attention<64>(tm_qkv, ap, seq, st);
