@@ -226,10 +226,38 @@ cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, cons
 }
 
 // LayerNorm + modulate launch: picks the register-resident row width (float4 per lane) for H.
+// Shared memory of the bulk-copy LayerNorm: 8 warps x slots row buffers, the cached shift and scale
+// vectors of one request (not for two-stream blocks), the barriers and the abort flag.
+constexpr size_t kLnTmaBudget = 224 * 1024;
+int ln_tma_slots(int H, bool from_bf16, bool cache_vectors) {
+  const size_t row_bytes = static_cast<size_t>(H) * (from_bf16 ? 2 : 4);
+  const size_t fixed = (cache_vectors ? static_cast<size_t>(H) * 8 : 0) + kLnTmaWarps * 4 * 8 + 16;
+  return static_cast<int>(std::min<size_t>(4, (kLnTmaBudget - fixed) / (kLnTmaWarps * row_bytes)));
+}
+size_t ln_tma_smem(int H, bool from_bf16, bool cache_vectors, int slots) {
+  const size_t row_bytes = static_cast<size_t>(H) * (from_bf16 ? 2 : 4);
+  return kLnTmaWarps * slots * (row_bytes + 8) + (cache_vectors ? static_cast<size_t>(H) * 8 : 0) + 16;
+}
+
+// LayerNorm + modulate launch: picks the register-resident row width (float4 per lane) for H.  Batches
+// of at least a few rows per SM take the bulk-copy kernel (one persistent CTA per SM), tiny ones the
+// plain one.  `num_sms` = 0 forces the plain kernel.
 template <bool kFromBf16, bool kOutFp8 = false>
 cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
                       long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st,
-                      long long kind_stride = 0, const RowGeom& geo = kNoGeom, float* row_scale = nullptr) {
+                      long long kind_stride = 0, const RowGeom& geo = kNoGeom, float* row_scale = nullptr,
+                      int num_sms = 0, int* status = nullptr) {
+  const bool cache_vectors = kind_stride == 0;
+  const int slots = ln_tma_slots(H, kFromBf16, cache_vectors);
+  if (num_sms > 0 && status && slots >= 1 && T >= 4 * num_sms) {
+    const int grid = std::min(num_sms, (T + kLnTmaWarps - 1) / kLnTmaWarps), block = kLnTmaWarps * 32;
+    const size_t smem = ln_tma_smem(H, kFromBf16, cache_vectors, slots);
+    const int cv = cache_vectors ? 1 : 0;
+    if (H <= 1024) ln_modulate_tma_kernel<kFromBf16, 8, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
+    else if (H <= 3072) ln_modulate_tma_kernel<kFromBf16, 24, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
+    else ln_modulate_tma_kernel<kFromBf16, 32, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
+    return cudaGetLastError();
+  }
   const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
   if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
   else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
@@ -363,10 +391,10 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
       if (fp8)
-        return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale)
-                      : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale);
-      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg)
-                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
+        return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
+                      : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status);
+      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status)
+                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
     }));
     // QKV projection
     GemmParams g{};
@@ -446,8 +474,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }));
     // LN2 + modulate
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      return fp8 ? launch_ln<false, true>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale)
-                 : launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg);
+      return fp8 ? launch_ln<false, true>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
+                 : launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
     }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};
@@ -584,6 +612,13 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 1024>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32Silu>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32>), mod_smem_bytes(kMaxCondDim));
+  {
+    auto ln_opt = [&](auto kernel) { opt_in(reinterpret_cast<const void*>(kernel), kLnTmaBudget); };
+    ln_opt(&ln_modulate_tma_kernel<false, 8, false>);  ln_opt(&ln_modulate_tma_kernel<false, 24, false>);  ln_opt(&ln_modulate_tma_kernel<false, 32, false>);
+    ln_opt(&ln_modulate_tma_kernel<true, 8, false>);   ln_opt(&ln_modulate_tma_kernel<true, 24, false>);   ln_opt(&ln_modulate_tma_kernel<true, 32, false>);
+    ln_opt(&ln_modulate_tma_kernel<false, 8, true>);   ln_opt(&ln_modulate_tma_kernel<false, 24, true>);   ln_opt(&ln_modulate_tma_kernel<false, 32, true>);
+    ln_opt(&ln_modulate_tma_kernel<true, 8, true>);    ln_opt(&ln_modulate_tma_kernel<true, 24, true>);    ln_opt(&ln_modulate_tma_kernel<true, 32, true>);
+  }
   if (e == cudaSuccess) {
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(sms & ~1); lc.blockDim = dim3(gemm_cfg::THREADS); lc.dynamicSmemBytes = gemm_cfg::SMEM_BYTES;
@@ -822,7 +857,8 @@ dit_status dit_ctx_poll_status(dit_ctx* ctx) {
   DIT_CUDA_TRY(ctx, cudaMemcpy(word, ctx->ws + ctx->lay.status, sizeof(word), cudaMemcpyDeviceToHost));
   if (word[0] == kStatusOk) return DIT_OK;
   DIT_CUDA_TRY(ctx, cudaMemset(ctx->ws + ctx->lay.status, 0, sizeof(word)));
-  return fail(ctx, DIT_ERR_TIMEOUT, "a bounded wait ran out in the %s kernel", word[0] == kStatusGemmTimeout ? "GEMM" : "attention");
+  return fail(ctx, DIT_ERR_TIMEOUT, "a bounded wait ran out in the %s kernel",
+              word[0] == kStatusGemmTimeout ? "GEMM" : (word[0] == kStatusAttnTimeout ? "attention" : "LayerNorm"));
 }
 
 dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t* rows, int64_t* cols, int32_t* elem_bytes) {
@@ -973,7 +1009,7 @@ dit_status final_impl(dit_ctx* ctx, const float* x, const SeqInfo& seq, const Sh
   if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM)) return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   DIT_CUDA_TRY(ctx, launch_small_linear<kModInCondSilu>(cond, ctx->ws + ctx->lay.sh_w_fa, ctx->at<float>(ctx->lay.sh_b_fa), nullptr,
                                                         modfin, nullptr, n, c.cond_dim, 2 * H, st));
-  DIT_CUDA_TRY(ctx, launch_ln<false>(x, nullptr, h, modfin, modfin + H, 2ll * H, T, H, c.ln_eps, seq, st));
+  DIT_CUDA_TRY(ctx, launch_ln<false>(x, nullptr, h, modfin, modfin + H, 2ll * H, T, H, c.ln_eps, seq, st, 0, kNoGeom, nullptr, ctx->num_sms, ctx->at<int>(ctx->lay.status)));
   GemmParams g{};
   g.status = ctx->at<int>(ctx->lay.status);
   g.M = T; g.N = DIT_PATCH_DIM; g.K = H;

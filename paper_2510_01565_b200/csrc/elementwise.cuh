@@ -2,6 +2,7 @@
 // and the one-off weight re-layout done at load time.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace dit {
 
@@ -143,17 +144,13 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 // ------------------------------------------------------------------------------------------------
 constexpr int kLnWarps = 4;
 
-// kOutFp8: h is written as e4m3 codes (1 byte per element, `h` then points at bytes) with one scale per
-// row, largest magnitude of the row -> 448; the scale goes to row_scale[row].
-template <bool kFromBf16, int kLnMaxVec, bool kOutFp8 = false>
-__global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVec <= 24 ? 4 : 3)))
-ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
-                   const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
-                   int T, int H, float eps, const __grid_constant__ SeqInfo seq,
-                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale) {
-  const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= T) return;
+// One row by one warp.  `src` points at the row's input (fp32, or bf16 with kFromBf16), in global or
+// shared memory.  kOutFp8: h is written as e4m3 codes (1 byte per element, `h` then points at bytes) with
+// one scale per row, largest magnitude of the row -> 448; the scale goes to row_scale[row].
+template <bool kFromBf16, int kLnMaxVec, bool kOutFp8>
+__device__ __forceinline__ void ln_modulate_row(const void* src, int row, int lane, float* __restrict__ stream_out,
+                                                __half* __restrict__ h, const float4* sh, const float4* sc, int H,
+                                                float eps, float* __restrict__ row_scale) {
   const int nvec = H >> 2;
   float4 v[kLnMaxVec];
   float sum = 0.f;
@@ -162,12 +159,12 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
     const int idx = i * 32 + lane;
     if (idx < nvec) {
       if (kFromBf16) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(xin) + static_cast<size_t>(row) * H) + idx);
+        const uint2 raw = *(reinterpret_cast<const uint2*>(src) + idx);
         v[i] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
                            __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
         reinterpret_cast<float4*>(stream_out + static_cast<size_t>(row) * H)[idx] = v[i];
       } else {
-        v[i] = reinterpret_cast<const float4*>(static_cast<const float*>(xin) + static_cast<size_t>(row) * H)[idx];
+        v[i] = reinterpret_cast<const float4*>(src)[idx];
       }
       sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
     }
@@ -186,18 +183,13 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
   const float rstd = rsqrtf(sq / static_cast<float>(H) + eps);
-  const int req = find_request(seq, row);
-  // two-stream blocks: text tokens take the text stream's vectors, kind_stride floats further on
-  const long long voff = req * req_stride + (kind_stride ? row_kind(seq, geo, req, row) * kind_stride : 0);
-  const float4* sh = reinterpret_cast<const float4*>(shift0 + voff);
-  const float4* sc = reinterpret_cast<const float4*>(scale0 + voff);
   if (kOutFp8) {
     float amax = 0.f;
 #pragma unroll
     for (int i = 0; i < kLnMaxVec; ++i) {
       const int idx = i * 32 + lane;
       if (idx < nvec) {
-        const float4 s1 = __ldg(sc + idx), s0 = __ldg(sh + idx);
+        const float4 s1 = sc[idx], s0 = sh[idx];
         v[i].x = (v[i].x - mean) * rstd * (1.f + s1.x) + s0.x;
         v[i].y = (v[i].y - mean) * rstd * (1.f + s1.y) + s0.y;
         v[i].z = (v[i].z - mean) * rstd * (1.f + s1.z) + s0.z;
@@ -226,7 +218,7 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
   for (int i = 0; i < kLnMaxVec; ++i) {
     const int idx = i * 32 + lane;
     if (idx < nvec) {
-      const float4 s1 = __ldg(sc + idx), s0 = __ldg(sh + idx);
+      const float4 s1 = sc[idx], s0 = sh[idx];
       const float a = (v[i].x - mean) * rstd * (1.f + s1.x) + s0.x;
       const float b = (v[i].y - mean) * rstd * (1.f + s1.y) + s0.y;
       const float c = (v[i].z - mean) * rstd * (1.f + s1.z) + s0.z;
@@ -235,6 +227,111 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
       dst[idx] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     }
   }
+}
+
+// Offset (floats) of the modulation vectors of `row`: its request's, and for two-stream blocks
+// (kind_stride != 0) the text stream's set for text tokens, kind_stride floats further on.
+__device__ __forceinline__ long long ln_vector_offset(const SeqInfo& seq, const RowGeom& geo, int row, long long req_stride,
+                                                      long long kind_stride) {
+  const int req = find_request(seq, row);
+  return req * req_stride + (kind_stride ? row_kind(seq, geo, req, row) * kind_stride : 0);
+}
+
+template <bool kFromBf16, int kLnMaxVec, bool kOutFp8 = false>
+__global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVec <= 24 ? 4 : 3)))
+ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
+                   const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
+                   int T, int H, float eps, const __grid_constant__ SeqInfo seq,
+                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale) {
+  const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= T) return;
+  const uint8_t* src = static_cast<const uint8_t*>(xin) + static_cast<size_t>(row) * H * (kFromBf16 ? 2 : 4);
+  const long long voff = ln_vector_offset(seq, geo, row, req_stride, kind_stride);
+  ln_modulate_row<kFromBf16, kLnMaxVec, kOutFp8>(src, row, lane, stream_out, h, reinterpret_cast<const float4*>(shift0 + voff),
+                                                 reinterpret_cast<const float4*>(scale0 + voff), H, eps, row_scale);
+}
+
+// The same rows fed by bulk copies.  Per-thread loads keep at most a few tens of KB in flight per SM
+// (they go through the L1's request tracking), which holds the kernel above at about half of the
+// HBM bandwidth; here every warp owns `slots` row buffers in shared memory that its lane 0 fills with
+// cp.async.bulk (one copy per row), so an SM has 8 x slots rows in flight.  A warp waits for a row,
+// processes it as above from shared memory and refills the buffer with its next row.
+// Persistent grid: CTA c owns the contiguous rows [c * chunk, (c + 1) * chunk), its warps take them
+// in turn.  Contiguous rows mostly share a request, so the CTA also keeps that request's shift and
+// scale vectors in shared memory (`cache_vectors`; with only 8 warps per SM their global loads would
+// otherwise sit on the critical path) and reloads them when its rows move on to the next request.
+constexpr int kLnTmaWarps = 8;
+
+template <bool kFromBf16, int kLnMaxVec, bool kOutFp8 = false>
+__global__ void __launch_bounds__(kLnTmaWarps * 32, 1)
+ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
+                       const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
+                       int T, int H, float eps, const __grid_constant__ SeqInfo seq,
+                       long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale,
+                       int slots, int cache_vectors, int* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t ln_smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t row_bytes = static_cast<uint32_t>(H) * (kFromBf16 ? 2u : 4u);
+  uint8_t* my_rows = ln_smem + static_cast<size_t>(warp) * slots * row_bytes;
+  uint8_t* after_rows = ln_smem + static_cast<size_t>(kLnTmaWarps) * slots * row_bytes;
+  float4* s_shift = reinterpret_cast<float4*>(after_rows);                     // [H] then scale [H] when cached
+  float4* s_scale = s_shift + (H >> 2);
+  uint8_t* after_vec = after_rows + (cache_vectors ? static_cast<size_t>(H) * 8 : 0);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(after_vec) + warp * slots;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(after_vec + kLnTmaWarps * slots * 8);
+  if (threadIdx.x == 0) *abort_flag = 0;
+  if (lane == 0) {
+    for (int s = 0; s < slots; ++s) mbar_init(smem_u32(bars + s), 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const int chunk = (T + gridDim.x - 1) / gridDim.x;
+  const int r0 = blockIdx.x * chunk, r1 = min(T, r0 + chunk);
+  auto fetch = [&](int row, int slot) {       // lane 0 only
+    mbar_arrive_expect_tx(smem_u32(bars + slot), row_bytes);
+    bulk_load(smem_u32(my_rows + static_cast<size_t>(slot) * row_bytes),
+              static_cast<const uint8_t*>(xin) + static_cast<size_t>(row) * row_bytes, row_bytes, smem_u32(bars + slot));
+  };
+  if (lane == 0)
+    for (int s = 0; s < slots; ++s)
+      if (r0 + warp + s * kLnTmaWarps < r1) fetch(r0 + warp + s * kLnTmaWarps, s);
+  int slot = 0; uint32_t phase = 0;
+  bool ok = true;
+  int row = r0 + warp;
+  // segments of the chunk that share one set of modulation vectors
+  for (int seg0 = r0; seg0 < r1;) {
+    int seg1 = r1;
+    if (cache_vectors) {
+      const int req = find_request(seq, seg0);
+      seg1 = min(r1, seq.cu[req + 1]);
+      __syncthreads();                              // every warp is done with the previous vectors
+      const float4* gsh = reinterpret_cast<const float4*>(shift0 + req * req_stride);
+      const float4* gsc = reinterpret_cast<const float4*>(scale0 + req * req_stride);
+      for (int i = threadIdx.x; i < (H >> 2); i += kLnTmaWarps * 32) { s_shift[i] = __ldg(gsh + i); s_scale[i] = __ldg(gsc + i); }
+      __syncthreads();
+    }
+    for (; row < seg1; row += kLnTmaWarps) {
+      if (ok && !__all_sync(0xffffffffu, mbar_wait(smem_u32(bars + slot), phase, abort_flag))) ok = false;
+      if (ok) {
+        const float4 *sh = s_shift, *sc = s_scale;
+        if (!cache_vectors) {
+          const long long voff = ln_vector_offset(seq, geo, row, req_stride, kind_stride);
+          sh = reinterpret_cast<const float4*>(shift0 + voff);
+          sc = reinterpret_cast<const float4*>(scale0 + voff);
+        }
+        ln_modulate_row<kFromBf16, kLnMaxVec, kOutFp8>(my_rows + static_cast<size_t>(slot) * row_bytes, row, lane, stream_out, h,
+                                                       sh, sc, H, eps, row_scale);
+        __syncwarp();                               // every lane has read the buffer: refill it
+        const int next = row + slots * kLnTmaWarps;
+        if (lane == 0 && next < r1) fetch(next, slot);
+        if (++slot == slots) { slot = 0; phase ^= 1u; }
+      }
+    }
+    seg0 = seg1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicMax(status, kStatusLnTimeout);
 }
 
 // ------------------------------------------------------------------------------------------------
