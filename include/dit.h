@@ -173,7 +173,7 @@ dit_status dit_pack_tokens(dit_ctx *ctx, const void *const *per_request_tokens, 
                            int32_t n, void *packed_tokens, void *stream);
 
 /* One denoising step: blocks 0..n_blocks-1 over the packed batch.
- *   packed_tokens           device [T, H] bf16, T = sum of lens; request r owns rows
+ *   packed_tokens           device [T, H] bf16, 16-byte aligned, T = sum of lens; request r owns rows
  *                           [cu[r], cu[r+1]) in input order
  *   per_request_token_lens  HOST [n_requests] int32, each >= 1; read before the call returns
  *   per_request_cond        device [n_requests, C] bf16; row r conditions request r
@@ -291,7 +291,7 @@ dit_status dit_timestep_cond(dit_ctx *ctx, const dit_request *requests, int32_t 
 dit_status dit_embed_latents(dit_ctx *ctx, const float *latents, const void *text_tokens,
                              const dit_request *requests, int32_t n, void *packed_tokens, void *stream);
 
-/* x [T, H] fp32 (device; the output of dit_step_forward), cond [n, C] bf16 (device) -> velocity. */
+/* x [T, H] fp32 (device, 16-byte aligned; the output of dit_step_forward), cond [n, C] bf16 (device) -> velocity. */
 dit_status dit_final_layer(dit_ctx *ctx, const float *x, const dit_request *requests, int32_t n,
                            const void *cond, float *velocity, void *stream);
 

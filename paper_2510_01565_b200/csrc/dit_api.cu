@@ -827,6 +827,8 @@ dit_status dit_step_forward(dit_ctx* ctx, const void* packed_tokens, const int32
                             int32_t n_blocks, float* out, void* stream) {
   dit_status s = check_step_args(ctx, packed_tokens, lens, n, cond, n_blocks, out);
   if (s != DIT_OK || n == 0) return s;
+  if (reinterpret_cast<uintptr_t>(packed_tokens) % 16 || reinterpret_cast<uintptr_t>(out) % 16)
+    return fail(ctx, DIT_ERR_INVALID_ARG, "packed_tokens and out must be 16-byte aligned");
   return step_impl(ctx, packed_tokens, lens, n, cond, n_blocks, out, static_cast<cudaStream_t>(stream));
 }
 
@@ -1141,6 +1143,8 @@ dit_status dit_step_forward_requests(dit_ctx* ctx, const void* packed_tokens, co
   for (int r = 0; r < n; ++r) lens[r] = seq.cu[r + 1] - seq.cu[r];
   s = check_step_args(ctx, packed_tokens, lens, n, cond, n_blocks, out);
   if (s != DIT_OK) return s;
+  if (reinterpret_cast<uintptr_t>(packed_tokens) % 16 || reinterpret_cast<uintptr_t>(out) % 16)
+    return fail(ctx, DIT_ERR_INVALID_ARG, "packed_tokens and out must be 16-byte aligned");
   const RowGeom geo = geom_of(info);
   return step_impl(ctx, packed_tokens, lens, n, cond, n_blocks, out, static_cast<cudaStream_t>(stream), &geo);
 }
