@@ -1106,6 +1106,7 @@ dit_status dit_final_layer(dit_ctx* ctx, const float* x, const dit_request* reqs
   dit_status s = check_shell_args(ctx, reqs, n);
   if (s != DIT_OK || n == 0) return s;
   if (!x || !cond || !velocity) return fail(ctx, DIT_ERR_INVALID_ARG, "NULL pointer argument");
+  if (reinterpret_cast<uintptr_t>(x) % 16) return fail(ctx, DIT_ERR_INVALID_ARG, "x must be 16-byte aligned");
   SeqInfo seq{}; ShellInfo info{};
   s = build_shell(ctx, reqs, n, nullptr, &seq, &info);
   if (s != DIT_OK) return s;
