@@ -197,6 +197,38 @@ def test_sixty_four_requests(B):
     run.close()
 
 
+def test_many_short_requests_in_a_long_batch(B):
+    # 48 requests of 17..40 tokens: about a thousand packed rows, so the LayerNorm kernel that streams
+    # rows through shared memory runs (it keeps one request's modulation vectors per CTA and must reload
+    # them several times inside each CTA's chunk of rows), as do several GEMM row tiles that mix requests
+    rng = np.random.default_rng(6)
+    reqs = [(16 * int(rng.integers(1, 3)), 16 * int(rng.integers(1, 3)), int(rng.integers(13, 24))) for _ in range(48)]
+    wl = W.make_custom("short", W.SMALL, 2, reqs, seed=6)
+    assert wl.total_tokens > 4 * 148 + 100
+    run = DeviceRun(B, wl, max_requests=48)
+    out = run.packed()
+    ref = oracle_requests(wl, range(48))
+    for r in range(48):
+        check_request(run, out, r, ref[r])
+    check_packed_equals_alone(run, out, requests=[0, 23, 47])
+    run.close()
+
+
+def test_widest_hidden_size(B):
+    # hidden 4096 (the largest the library takes): 16 KB rows leave one row buffer per warp in the
+    # streaming LayerNorm kernel, and the GEMMs get a K that is not a multiple of 3072
+    dims = W.ModelDims(hidden=4096, n_heads=32, head_dim=128, mlp_hidden=4096, cond_dim=256)
+    wl = W.make_custom("wide", dims, 1, [(256, 256, 384), (64, 64, 0)], seed=8)
+    assert wl.total_tokens >= 4 * 148
+    run = DeviceRun(B, wl)
+    out = run.packed()
+    ref = oracle_requests(wl, [0, 1])
+    check_request(run, out, 0, ref[0])
+    check_request(run, out, 1, ref[1])
+    check_packed_equals_alone(run, out)
+    run.close()
+
+
 def test_zero_gate_returns_input_exactly(B):
     wl = W.make_custom("zerogate", W.SMALL, 2, [(256, 256, 5), (64, 64, 0)], seed=6, timestep_cond=False)
     H = wl.dims.hidden
