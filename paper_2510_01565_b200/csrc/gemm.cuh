@@ -356,10 +356,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
           }
           __syncwarp();                        // staging buffer is reused by the next chunk
-        } else if (row_ok) {
-          const bool full = (col0 + 32 <= p.N);
-          __half* dst = p.out16 + static_cast<size_t>(row) * (p.ld16 ? p.ld16 : p.N) + col0;
+        } else {
+          const bool full = (col0 + 32 <= p.N);            // warp-uniform
+          const int ld = p.ld16 ? p.ld16 : p.N;
           if (full) {
+            // fp16 results go through shared memory so that a store instruction covers 64 contiguous
+            // bytes of each of 8 rows (whole sectors) instead of 16 bytes of each of 32 rows
+            uint8_t* stb = reinterpret_cast<uint8_t*>(epi_stage + (warp - 2) * EPI_STAGE_FLOATS);
+            uint4* srow = reinterpret_cast<uint4*>(stb + lane * 80);
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
               uint32_t w[4];
@@ -374,9 +378,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const __half2 hh = __floats2half2_rn(a, b);
                 w[h] = *reinterpret_cast<const uint32_t*>(&hh);
               }
-              *(reinterpret_cast<uint4*>(dst) + v) = make_uint4(w[0], w[1], w[2], w[3]);
+              srow[v] = make_uint4(w[0], w[1], w[2], w[3]);
             }
-          } else {
+            __syncwarp();
+            const unsigned ok_rows = __ballot_sync(0xffffffffu, row_ok);
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int rr = it * 8 + (lane >> 2), part = lane & 3;
+              if ((ok_rows >> rr) & 1u) {
+                const uint4 val = *reinterpret_cast<const uint4*>(stb + rr * 80 + part * 16);
+                *reinterpret_cast<uint4*>(p.out16 + static_cast<size_t>(m0 + quarter * 32 + rr) * ld + col0 + part * 8) = val;
+              }
+            }
+            __syncwarp();                      // staging buffer is reused by the next chunk
+          } else if (row_ok) {
+            __half* dst = p.out16 + static_cast<size_t>(row) * ld + col0;
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               if (col0 + i < p.N) {
