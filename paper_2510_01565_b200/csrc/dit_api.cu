@@ -126,6 +126,8 @@ struct BlockState {
 
 }  // namespace
 
+constexpr int kHostOutSlices = 4;
+
 struct dit_ctx {
   dit_config cfg;
   Layout lay;
@@ -142,6 +144,10 @@ struct dit_ctx {
   char err[256];
   // optional per-kernel timing (CUDA events recorded around every launch of a step)
   bool timing;
+  // dit_step_forward_host: the output goes back to the host in row slices while the last GEMM still runs
+  cudaStream_t copy_stream;
+  cudaEvent_t slice_done[kHostOutSlices], copies_done, tok_ready[kHostOutSlices];
+  bool host_copied;                        // the last step_impl call sent its output to the host itself
   std::vector<cudaEvent_t> ev_pool;        // pairs: [2i] start, [2i+1] stop
   std::vector<int> ev_kind;                // kind of pair i
   size_t ev_used;                          // pairs recorded since the last read
@@ -246,22 +252,22 @@ template <bool kFromBf16, bool kOutFp8 = false>
 cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
                       long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st,
                       long long kind_stride = 0, const RowGeom& geo = kNoGeom, float* row_scale = nullptr,
-                      int num_sms = 0, int* status = nullptr) {
+                      int num_sms = 0, int* status = nullptr, int row0 = 0) {
   const bool cache_vectors = kind_stride == 0;
   const int slots = ln_tma_slots(H, kFromBf16, cache_vectors);
   if (num_sms > 0 && status && slots >= 1 && T >= 4 * num_sms) {
     const int grid = std::min(num_sms, (T + kLnTmaWarps - 1) / kLnTmaWarps), block = kLnTmaWarps * 32;
     const size_t smem = ln_tma_smem(H, kFromBf16, cache_vectors, slots);
     const int cv = cache_vectors ? 1 : 0;
-    if (H <= 1024) ln_modulate_tma_kernel<kFromBf16, 8, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
-    else if (H <= 3072) ln_modulate_tma_kernel<kFromBf16, 24, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
-    else ln_modulate_tma_kernel<kFromBf16, 32, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status);
+    if (H <= 1024) ln_modulate_tma_kernel<kFromBf16, 8, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
+    else if (H <= 3072) ln_modulate_tma_kernel<kFromBf16, 24, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
+    else ln_modulate_tma_kernel<kFromBf16, 32, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
     return cudaGetLastError();
   }
   const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
-  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
-  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
-  else ln_modulate_kernel<kFromBf16, 32, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale);
+  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
+  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
+  else ln_modulate_kernel<kFromBf16, 32, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
   return cudaGetLastError();
 }
 
@@ -282,8 +288,12 @@ cudaError_t launch_modulation(const ModParams& mp, int num_sms, size_t smem, cud
 }
 
 // `geo` (image geometry of the requests) is needed by the rotary term only; NULL otherwise.
+// `host_out` (dit_step_forward_host): the last GEMM runs in row slices and every finished slice of `out` is
+// copied to the host on the context's copy stream while the next slice computes.  `tokens_in_slices`: the
+// tokens are being copied in by the same slices (events tok_ready) and block 0 starts on each as it lands.
 dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
-                     float* out, cudaStream_t st, const RowGeom* geo = nullptr) {
+                     float* out, cudaStream_t st, const RowGeom* geo = nullptr, float* host_out = nullptr,
+                     bool tokens_in_slices = false) {
   const dit_config& c = ctx->cfg;
   SeqInfo seq{};
   if (!build_seq(lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
@@ -340,6 +350,35 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     return cudaEventRecord(ctx->ev_pool[2 * i + 1], st);
   };
 
+  // The gated-residual GEMM that writes `out`, sliced by rows when the result goes to the host.  A slice is a
+  // whole number of 256-row tiles; every output element is computed exactly as in the unsliced launch.
+  auto last_gemm = [&](const __half* a_ptr, int K, const CUtensorMap& tmA_full, const CUtensorMap& tmB, const GemmParams& g) -> dit_status {
+    if (!host_out) {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tmA_full, tmB, g, seq, st); }));
+      return DIT_OK;
+    }
+    const int tile_rows = 2 * gemm_cfg::BM;
+    const int per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;   // rows per slice
+    for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
+      const int rows = std::min(per, T - r0);
+      CUtensorMap tmA;
+      if (!make_map(ctx, &tmA, a_ptr + static_cast<size_t>(r0) * K, K, rows, gemm_cfg::BM))
+        return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+      GemmParams q = g;
+      q.M = rows; q.row0 = r0;
+      q.resid = g.resid + static_cast<size_t>(r0) * g.N;
+      q.out32 = g.out32 + static_cast<size_t>(r0) * g.N;
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tmA, tmB, q, seq, st); }));
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->slice_done[sidx], st));
+      DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->slice_done[sidx], 0));
+      DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out + static_cast<size_t>(r0) * g.N, g.out32 + static_cast<size_t>(r0) * g.N,
+                                        static_cast<size_t>(rows) * g.N * 4, cudaMemcpyDeviceToHost, ctx->copy_stream));
+    }
+    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, ctx->copy_stream));
+    ctx->host_copied = true;
+    return DIT_OK;
+  };
+
   {  // adaLN modulation vectors of every block
     ModParams mp{};
     mp.cond = static_cast<const __nv_bfloat16*>(cond);
@@ -388,15 +427,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       gp.bias2 = reinterpret_cast<const float*>(wt + bias_off);
       gp.gate_kind_stride = ks;
     };
-    // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream)
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
-      if (fp8)
-        return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
-                      : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status);
-      return b == 0 ? launch_ln<true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status)
-                    : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
-    }));
-    // QKV projection
+    // LN1 + modulate (block 0 also widens the bf16 tokens into the fp32 residual stream) and the QKV projection,
+    // over packed rows [r0, r0 + rows): the whole batch, or one slice of it while the host's tokens still arrive
     GemmParams g{};
     g.status = status;
     g.M = T; g.N = 3 * H; g.K = H;
@@ -413,22 +445,58 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
         g.k_norm2 = reinterpret_cast<const float*>(wt + ctx->lay.blk.k_norm);
       }
       if (c.flags & DIT_FLAG_ROPE_2D) g.rope_theta = ctx->at<float>(ctx->lay.rope_theta);
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+    }
+    auto ln1_qkv = [&](int r0, int rows, const CUtensorMap& tmA) -> dit_status {
+      const size_t e0 = static_cast<size_t>(r0) * H;      // first element of the slice in a [T, H] buffer
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
         if (fp8)
-          return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg)
-                                   : launch_gemm<kEpiQkvF16, 64, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg);
-        if (dual)
-          return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
-                                   : launch_gemm<kEpiQkvF16, 64, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv);
-        return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg)
-                                 : launch_gemm<kEpiQkvF16, 64>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg);
+          return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
+                        : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status);
+        return b == 0 ? launch_ln<true>(static_cast<const __nv_bfloat16*>(tokens) + e0, stream + e0, h + e0, modb, modb + H, req_stride, rows, H,
+                                        c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status, r0)
+                      : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
       }));
+      GemmParams q = g;
+      q.M = rows; q.row0 = r0; q.out16 = qkv + static_cast<size_t>(r0) * 3 * H;
+      if (qk_variant) {
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+          if (fp8)
+            return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, false, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg)
+                                     : launch_gemm<kEpiQkvF16, 64, false, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg);
+          if (dual)
+            return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg, &bt.tm_qkv)
+                                     : launch_gemm<kEpiQkvF16, 64, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg, &bt.tm_qkv);
+          return c.head_dim == 128 ? launch_gemm<kEpiQkvF16, 128>(ctx, tmA, bs.tm_qkv, q, seq, st, rg)
+                                   : launch_gemm<kEpiQkvF16, 64>(ctx, tmA, bs.tm_qkv, q, seq, st, rg);
+        }));
+      } else {
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
+          if (fp8) return launch_gemm<kEpiBiasF16, 0, false, true>(ctx, tmA, bs.tm_qkv, q, seq, st);
+          return dual ? launch_gemm<kEpiBiasF16, 0, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg, &bt.tm_qkv)
+                      : launch_gemm<kEpiBiasF16>(ctx, tmA, bs.tm_qkv, q, seq, st);
+        }));
+      }
+      return DIT_OK;
+    };
+    if (b == 0 && tokens_in_slices && !fp8 && !dual) {
+      // dit_step_forward_host: the tokens are on their way in row slices on the copy stream; each slice is
+      // normalised and projected as soon as it has landed
+      const int tile_rows = 2 * gemm_cfg::BM;
+      const int per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;
+      for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
+        const int rows = std::min(per, T - r0);
+        DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->tok_ready[sidx], 0));
+        CUtensorMap tmA;
+        if (!make_map(ctx, &tmA, h + static_cast<size_t>(r0) * H, H, rows, gemm_cfg::BM))
+          return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+        const dit_status ls = ln1_qkv(r0, rows, tmA);
+        if (ls != DIT_OK) return ls;
+      }
     } else {
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
-        if (fp8) return launch_gemm<kEpiBiasF16, 0, false, true>(ctx, tm_h, bs.tm_qkv, g, seq, st);
-        return dual ? launch_gemm<kEpiBiasF16, 0, true>(ctx, tm_h, bs.tm_qkv, g, seq, st, rg, &bt.tm_qkv)
-                    : launch_gemm<kEpiBiasF16>(ctx, tm_h, bs.tm_qkv, g, seq, st);
-      }));
+      if (b == 0 && tokens_in_slices)
+        for (int sidx = 0; sidx < kHostOutSlices; ++sidx) DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->tok_ready[sidx], 0));
+      const dit_status ls = ln1_qkv(0, T, tm_h);
+      if (ls != DIT_OK) return ls;
     }
     // attention (one pass over all tokens of a request, whatever their stream)
     AttnParams ap{};
@@ -457,7 +525,12 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
       g.resid = stream; g.out32 = last ? out : stream;
       g.gate = modb + 2 * H; g.gate_stride = req_stride;
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
+      if (last) {
+        const dit_status ls = last_gemm(cat, H + F, tm_cat, bs.tm_fc2, g);
+        if (ls != DIT_OK) return ls;
+      } else {
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
+      }
       continue;
     }
     // output projection + gate + residual
@@ -498,10 +571,15 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.resid = stream; g.out32 = last ? out : stream;
     g.gate = modb + 5 * H; g.gate_stride = req_stride;
     two_stream(g, ctx->lay.blk.b_fc2);
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] {
-      return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_u, bs.tm_fc2, g, seq, st, rg, &bt.tm_fc2)
-                  : launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st);
-    }));
+    if (last && !dual) {
+      const dit_status ls = last_gemm(u, F, tm_u, bs.tm_fc2, g);
+      if (ls != DIT_OK) return ls;
+    } else {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] {
+        return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_u, bs.tm_fc2, g, seq, st, rg, &bt.tm_fc2)
+                    : launch_gemm<kEpiGateResidF32>(ctx, tm_u, bs.tm_fc2, g, seq, st);
+      }));
+    }
   }
   ctx->last_launches = launches;
   ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
@@ -630,6 +708,14 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
     e = cudaOccupancyMaxActiveClusters(&clusters, reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16>), &lc);
     ctx->gemm_pairs = std::max(1, std::min(clusters, sms / 2));
   }
+  ctx->copy_stream = nullptr;
+  ctx->host_copied = false;
+  ctx->copies_done = nullptr;
+  for (int i = 0; i < kHostOutSlices; ++i) { ctx->slice_done[i] = nullptr; ctx->tok_ready[i] = nullptr; }
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+  for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->slice_done[i], cudaEventDisableTiming);
+  for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->tok_ready[i], cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->copies_done, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
   if (e == cudaSuccess) {
     // rotary pair frequencies of one axis group of n = (d - d/8) / 2 channels: 10000^(-2i/n), i < n/2
@@ -638,7 +724,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
     for (int i = 0; i < n_axis / 2; ++i) theta[i] = static_cast<float>(pow(10000.0, -2.0 * i / n_axis));
     e = cudaMemcpy(ctx->ws + lay.rope_theta, theta, sizeof(theta), cudaMemcpyHostToDevice);
   }
-  if (e != cudaSuccess) { delete[] ctx->blocks; delete ctx; return DIT_ERR_CUDA; }
+  if (e != cudaSuccess) { dit_ctx_destroy(ctx); return DIT_ERR_CUDA; }
   *out = ctx;
   return DIT_OK;
 }
@@ -646,6 +732,10 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
 dit_status dit_ctx_destroy(dit_ctx* ctx) {
   if (!ctx) return DIT_ERR_INVALID_ARG;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  for (int i = 0; i < kHostOutSlices; ++i) if (ctx->slice_done[i]) cudaEventDestroy(ctx->slice_done[i]);
+  for (int i = 0; i < kHostOutSlices; ++i) if (ctx->tok_ready[i]) cudaEventDestroy(ctx->tok_ready[i]);
+  if (ctx->copies_done) cudaEventDestroy(ctx->copies_done);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   delete[] ctx->blocks;
   delete ctx;
   return DIT_OK;
@@ -843,11 +933,29 @@ dit_status dit_step_forward_host(dit_ctx* ctx, const void* host_tokens, const in
   void* d_tok = ctx->ws + ctx->lay.stage_tokens;
   void* d_cond = ctx->ws + ctx->lay.stage_cond;
   float* d_out = ctx->at<float>(ctx->lay.stage_out);
-  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(d_tok, host_tokens, T * H * 2, cudaMemcpyHostToDevice, st));
+  // cond first (the modulation kernel needs nothing else), then the tokens in row slices on the copy stream:
+  // block 0 starts on a slice as soon as it has landed, the slices behind it overlap its work
   DIT_CUDA_TRY(ctx, cudaMemcpyAsync(d_cond, host_cond, n * C * 2, cudaMemcpyHostToDevice, st));
-  s = step_impl(ctx, d_tok, lens, n, d_cond, n_blocks, d_out, st);
+  {
+    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, st));                 // order the copy stream after earlier work on st
+    DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->copies_done, 0));
+    const size_t tile_rows = 2 * gemm_cfg::BM;
+    const size_t per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;
+    for (size_t sidx = 0, r0 = 0; sidx < static_cast<size_t>(kHostOutSlices); ++sidx, r0 += per) {
+      if (r0 < T) {
+        const size_t rows = std::min(per, T - r0);
+        DIT_CUDA_TRY(ctx, cudaMemcpyAsync(static_cast<uint8_t*>(d_tok) + r0 * H * 2, static_cast<const uint8_t*>(host_tokens) + r0 * H * 2,
+                                          rows * H * 2, cudaMemcpyHostToDevice, ctx->copy_stream));
+      }
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->tok_ready[sidx], ctx->copy_stream));
+    }
+  }
+  ctx->host_copied = false;
+  s = step_impl(ctx, d_tok, lens, n, d_cond, n_blocks, d_out, st, nullptr, host_out, true);
   if (s != DIT_OK) return s;
-  DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, d_out, T * H * 4, cudaMemcpyDeviceToHost, st));
+  // the output normally went back slice by slice on the copy stream (see step_impl): join it
+  if (ctx->host_copied) DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->copies_done, 0));
+  else DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, d_out, T * H * 4, cudaMemcpyDeviceToHost, st));
   DIT_CUDA_TRY(ctx, cudaStreamSynchronize(st));
   return DIT_OK;
 }

@@ -242,12 +242,14 @@ __global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVe
 ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
                    const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                    int T, int H, float eps, const __grid_constant__ SeqInfo seq,
-                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale) {
+                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale, int row0) {
+  // rows are local to the launch (a launch may cover a slice of the batch starting at packed row row0:
+  // the data pointers are already offset, only the request lookup needs the packed index)
   const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= T) return;
   const uint8_t* src = static_cast<const uint8_t*>(xin) + static_cast<size_t>(row) * H * (kFromBf16 ? 2 : 4);
-  const long long voff = ln_vector_offset(seq, geo, row, req_stride, kind_stride);
+  const long long voff = ln_vector_offset(seq, geo, row + row0, req_stride, kind_stride);
   ln_modulate_row<kFromBf16, kLnMaxVec, kOutFp8>(src, row, lane, stream_out, h, reinterpret_cast<const float4*>(shift0 + voff),
                                                  reinterpret_cast<const float4*>(scale0 + voff), H, eps, row_scale);
 }
@@ -269,7 +271,7 @@ ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_
                        const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                        int T, int H, float eps, const __grid_constant__ SeqInfo seq,
                        long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale,
-                       int slots, int cache_vectors, int* __restrict__ status) {
+                       int slots, int cache_vectors, int* __restrict__ status, int row0) {
   extern __shared__ __align__(128) uint8_t ln_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t row_bytes = static_cast<uint32_t>(H) * (kFromBf16 ? 2u : 4u);
@@ -303,8 +305,8 @@ ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_
   for (int seg0 = r0; seg0 < r1;) {
     int seg1 = r1;
     if (cache_vectors) {
-      const int req = find_request(seq, seg0);
-      seg1 = min(r1, seq.cu[req + 1]);
+      const int req = find_request(seq, seg0 + row0);
+      seg1 = min(r1, seq.cu[req + 1] - row0);
       __syncthreads();                              // every warp is done with the previous vectors
       const float4* gsh = reinterpret_cast<const float4*>(shift0 + req * req_stride);
       const float4* gsc = reinterpret_cast<const float4*>(scale0 + req * req_stride);
@@ -316,7 +318,7 @@ ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_
       if (ok) {
         const float4 *sh = s_shift, *sc = s_scale;
         if (!cache_vectors) {
-          const long long voff = ln_vector_offset(seq, geo, row, req_stride, kind_stride);
+          const long long voff = ln_vector_offset(seq, geo, row + row0, req_stride, kind_stride);
           sh = reinterpret_cast<const float4*>(shift0 + voff);
           sc = reinterpret_cast<const float4*>(scale0 + voff);
         }

@@ -39,6 +39,7 @@ struct GemmParams {
   const float* gate;        // gate vector of request 0 for this block; request r at gate + r * gate_stride
   long long gate_stride;
   int ld16;
+  int row0;                 // packed row index of row 0 of A / out (a launch may cover a slice of the batch's rows)
   int* status;              // device status word
   // kEpiQkvF16 only
   const float* q_norm;      // [HD] RMS-norm scale of the queries, NULL = no RMS-norm
@@ -206,10 +207,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int row = m0 + quarter * 32 + lane;
       // gated-residual epilogue: request of this lane's row, and whether the warp's rows share it
       int my_req = -1;
-      if ((EPI == kEpiGateResidF32 || DUAL) && row < p.M) my_req = find_request(seq, row);
+      if ((EPI == kEpiGateResidF32 || DUAL) && row < p.M) my_req = find_request(seq, row + p.row0);
       // two-stream launch: this pass stores only the rows of its own stream
       int my_kind = -1;
-      if (DUAL && row < p.M) my_kind = row_kind(seq, geo, my_req, row);
+      if (DUAL && row < p.M) my_kind = row_kind(seq, geo, my_req, row + p.row0);
       const bool row_ok = row < p.M && (!DUAL || my_kind == kind);
       const float sa = (FP8 && row < p.M) ? p.row_scale[row] : 1.0f;
       const float* bias = (DUAL && kind) ? p.bias2 : p.bias;
@@ -240,8 +241,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // patch row and column of this lane's token (text tokens and rows past M: (0, 0))
         int py = 0, px = 0;
         if (p.rope_theta && row_ok) {
-          const int rq = find_request(seq, row);
-          const int local = row - seq.cu[rq];
+          const int rq = find_request(seq, row + p.row0);
+          const int local = row + p.row0 - seq.cu[rq];
           if (local < geo.img_cu[rq + 1] - geo.img_cu[rq]) { py = local / geo.gw[rq]; px = local - py * geo.gw[rq]; }
         }
 #pragma unroll 1

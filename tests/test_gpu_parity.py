@@ -107,10 +107,21 @@ def test_cfg1_small_block_full_parity_and_taps(B):
 
 
 def test_cfg2_512_four_blocks(B):
+    import torch
     wl = W.make_workload("cfg2_512")
     run = DeviceRun(B, wl)
     out = run.packed()
     check_request(run, out, 0, oracle_requests(wl, [0])[0])
+    # the host-buffer entry point moves tokens in and the output out in row slices that overlap the
+    # first and the last kernels (1536 rows = 3 slices here): same bits as the device-buffer call
+    h_tok = torch.from_numpy(wl.packed_tokens().view(np.int16)).pin_memory()
+    h_cond = torch.from_numpy(wl.cond.view(np.int16)).pin_memory()
+    h_out = torch.full(out.shape, float("nan"), dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        run.ctx.dit_step_forward_host(h_tok, wl.token_lens, h_cond, wl.n_blocks, h_out)
+        assert torch.equal(h_out, out.cpu())
+        h_out.fill_(float("nan"))
+    run.ctx.dit_ctx_poll_status()
     run.close()
 
 
