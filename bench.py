@@ -368,6 +368,17 @@ def run_gpu(args):
                 "algorithmic_bytes": (T * H * 2 * 2 + 3 * H * H * 2 + T * 3 * H * 2 + H * H * 2 + T * H * 8 + T * H * 2 + H * F * 2
                                       + T * F * 2 * 2 + F * H * 2 + T * H * 8) / 4.0}
 
+    # the largest single kernel by time is attention: its own figure beside the GEMMs' (same peak; at d = 128
+    # its exponentials need as many special-function cycles as its MMAs need tensor cycles)
+    roofline_attention = None
+    if "attention" in kern:
+        a = kern["attention"]
+        roofline_attention = {"bound": "tensor", "kernel": "attention_tcgen05_kernel", "achieved": a["tflops"],
+                              "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                              "frac": a["tflops"] / peaks["bf16_tflops_sustained"], "avg_launch_ms": a["avg_ms"],
+                              "launches": a["launches"], "share_of_step": a["share"],
+                              "traffic": None}
+
     # ---------------------------------------------------------------- the oracle on the host cores
     run, n_img, desc = oracle_sample(wl)
     reps, t0 = 0, time.perf_counter()
@@ -388,7 +399,7 @@ def run_gpu(args):
                        "l2": "weights and activations of a step exceed L2 (126 MB); no flush"},
             "tflops": tflops, "frac_of_bf16_peak": tflops / peaks["bf16_tflops"],
             "frac_of_bf16_sustained": tflops / peaks["bf16_tflops_sustained"], "peaks": peaks,
-            "roofline": roofline, "kernels": kern, "cpu_baseline": cpu,
+            "roofline": roofline, "roofline_attention": roofline_attention, "kernels": kern, "cpu_baseline": cpu,
             "e2e": {"value": img_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "cuda_graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms, "value": replicas.whole_job_rate(wl.image_tokens, world, graph_ms), "unit": UNIT},
