@@ -606,6 +606,8 @@ dit_status check_step_args(dit_ctx* ctx, const void* tokens, const int32_t* lens
   if (n > ctx->cfg.max_requests) return fail(ctx, DIT_ERR_CAPACITY, "n_requests exceeds max_requests");
   if (n_blocks < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "n_blocks must be at least 1");
   if (n_blocks > ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "n_blocks exceeds max_blocks");
+  for (int b = 0; b < n_blocks; ++b)
+    if (!ctx->blocks[b].loaded) return fail(ctx, DIT_ERR_NOT_LOADED, "a block in [0, n_blocks) has no weights");
   long long total = 0;
   for (int r = 0; r < n; ++r) {
     if (lens[r] < 1) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
