@@ -138,6 +138,8 @@ struct dit_ctx {
   BlockState* blocks;
   bool shell_loaded;
   CUtensorMap tm_wout;                     // W_out^T, fp16 [kWoutRows, H]
+  CUtensorMap tm_wada;                     // every block's W_ada as one 3-D tensor [max_blocks, C, 6H] bf16, boxes of 10 x 256
+  bool tm_wada_ok;
   int64_t last_launches;
   int last_T, last_R, last_nb;
   bool last_parallel;                      // the last block of the last step was a parallel block
@@ -275,11 +277,22 @@ size_t mod_smem_bytes(int C) {   // activations [G][C], later reused for the sli
   return std::max<size_t>(static_cast<size_t>(kModReqGroup) * C, static_cast<size_t>(8) * kModThreads * kModReqGroup) * sizeof(float);
 }
 
-// adaLN modulation of all blocks: the widest column strip that still leaves about two CTAs per SM
+size_t mod_tma_smem_bytes(int C) {
+  return mod_tma_act_floats(C) * sizeof(float) + kModTmaRingBytes + 2 * kModTmaSlices * kModTmaStages * 8 + 16;
+}
+constexpr size_t kModTmaSmemMax = 224 * 1024;
+
+// adaLN modulation of all blocks.  With enough strips of 512 columns to give every SM about two CTAs, and
+// a cond width whose activations leave room for the ring, W_ada is streamed by bulk copies; otherwise the
+// register-load kernel runs with the widest column strip that still leaves about two CTAs per SM
 // (measured on the 8-block mixed step: 0.72 / 0.57 / 0.48 ms for 128 / 256 / 512 columns).
-cudaError_t launch_modulation(const ModParams& mp, int num_sms, size_t smem, cudaStream_t st) {
+cudaError_t launch_modulation(const ModParams& mp, int num_sms, size_t smem, cudaStream_t st, int* status, const CUtensorMap* tmW) {
   auto ctas = [&](int cols) { return mp.NB * ((mp.N6 + cols - 1) / cols); };
   const int enough = 3 * num_sms / 2;
+  if (status && tmW && ctas(kModTmaCols) >= enough && mod_tma_smem_bytes(mp.C) <= kModTmaSmemMax) {
+    modulation_tma_kernel<<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C), st>>>(*tmW, mp, status);
+    return cudaGetLastError();
+  }
   if (ctas(1024) >= enough) modulation_kernel<kModInCondSilu, 1024><<<ctas(1024), kModThreads, smem, st>>>(mp);
   else if (ctas(512) >= enough) modulation_kernel<kModInCondSilu, 512><<<ctas(512), kModThreads, smem, st>>>(mp);
   else if (ctas(256) >= enough) modulation_kernel<kModInCondSilu, 256><<<ctas(256), kModThreads, smem, st>>>(mp);
@@ -387,7 +400,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     mp.w_block_stride = static_cast<long long>(ctx->lay.blk.bytes / 2);
     mp.b_block_stride = static_cast<long long>(ctx->lay.blk.bytes / 4);
     mp.mod = mod; mp.R = n; mp.C = c.cond_dim; mp.N6 = 6 * H; mp.NB = n_blocks;
-    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_MODULATION, [&] { return launch_modulation(mp, ctx->num_sms, mod_smem_bytes(c.cond_dim), st); }));
+    DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_MODULATION, [&] { return launch_modulation(mp, ctx->num_sms, mod_smem_bytes(c.cond_dim), st, status, ctx->tm_wada_ok ? &ctx->tm_wada : nullptr); }));
   }
 
   // two-stream blocks: validate the pairing and list the row tiles of each stream once per step
@@ -690,6 +703,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 256>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 512>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 1024>), mod_smem_bytes(kMaxCondDim));
+  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel), kModTmaSmemMax);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32Silu>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32>), mod_smem_bytes(kMaxCondDim));
   {
@@ -714,6 +728,15 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->host_copied = false;
   ctx->copies_done = nullptr;
   for (int i = 0; i < kHostOutSlices; ++i) { ctx->slice_done[i] = nullptr; ctx->tok_ready[i] = nullptr; }
+  {
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(6) * cfg->hidden, static_cast<cuuint64_t>(cfg->cond_dim), static_cast<cuuint64_t>(cfg->max_blocks)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(6) * cfg->hidden * 2, static_cast<cuuint64_t>(lay.blk.bytes)};
+    const cuuint32_t box[3] = {256, kModTmaRows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    ctx->tm_wada_ok = ctx->encode(&ctx->tm_wada, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ctx->ws + lay.weights + lay.blk.w_ada, dims, strides, box,
+                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
   for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->slice_done[i], cudaEventDisableTiming);
   for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->tok_ready[i], cudaEventDisableTiming);
@@ -970,7 +993,7 @@ dit_status dit_ctx_poll_status(dit_ctx* ctx) {
   if (word[0] == kStatusOk) return DIT_OK;
   DIT_CUDA_TRY(ctx, cudaMemset(ctx->ws + ctx->lay.status, 0, sizeof(word)));
   return fail(ctx, DIT_ERR_TIMEOUT, "a bounded wait ran out in the %s kernel",
-              word[0] == kStatusGemmTimeout ? "GEMM" : (word[0] == kStatusAttnTimeout ? "attention" : "LayerNorm"));
+              word[0] == kStatusGemmTimeout ? "GEMM" : (word[0] == kStatusAttnTimeout ? "attention" : (word[0] == kStatusLnTimeout ? "LayerNorm" : "modulation")));
 }
 
 dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t* rows, int64_t* cols, int32_t* elem_bytes) {

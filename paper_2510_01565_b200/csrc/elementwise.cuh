@@ -134,6 +134,153 @@ __global__ void __launch_bounds__(kModThreads) modulation_kernel(const ModParams
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same modulation with W_ada streamed by TMA (for the adaLN modulation of a whole stack,
+// kModInCondSilu only).  Per-thread loads keep about 48 KB in flight per SM; here a CTA owns a strip of
+// 512 columns of one block; its four slices of the C range (two compute warps each) each have a
+// two-stage ring of 15-row groups, 120 KB in flight per SM, refilled by a ninth warp that does nothing
+// else (lane s serves slice s), so a compute warp only ever waits for data.  A group arrives as two
+// boxes of 256 columns x 15 rows of a 3-D tensor map over every block's W_ada (measured: 10-row groups
+// in three stages 0.38 ms, 6-row groups in five 0.40 ms, 15-row groups in two 0.36 ms; one 1 KB bulk
+// copy per row 0.56 ms; the register-load kernel 0.48-0.51 ms).  The activations sit in shared memory
+// request-minor ([c][8]) so that a row costs two 16-byte loads, and the products use packed fp32
+// pairs.  Summation order: that of modulation_kernel<.., 512>.
+// ------------------------------------------------------------------------------------------------
+constexpr int kModTmaCols = 512, kModTmaSlices = 4, kModTmaStages = 2, kModTmaRows = 15;
+constexpr int kModTmaComputeThreads = 256, kModTmaThreads = kModTmaComputeThreads + 32;
+constexpr int kModTmaRingBytes = kModTmaSlices * kModTmaStages * kModTmaRows * kModTmaCols * 2;
+
+__host__ __device__ inline size_t mod_tma_act_floats(int C) {      // activations [C][G], later the slice partials
+  const size_t a = static_cast<size_t>(kModReqGroup) * C, b = static_cast<size_t>(kModTmaSlices) * kModReqGroup * kModTmaCols;
+  return a > b ? a : b;
+}
+
+__global__ void __launch_bounds__(kModTmaThreads, 1)
+modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p, int* __restrict__ status) {
+  static_assert(kModReqGroup == 8, "the activation layout below packs 8 requests per row");
+  extern __shared__ __align__(128) uint8_t mod_smem[];
+  float* s_act = reinterpret_cast<float*>(mod_smem);               // [C][8]
+  float* s_part = s_act;
+  uint8_t* ring = mod_smem + mod_tma_act_floats(p.C) * sizeof(float);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + kModTmaRingBytes);      // full[slice][stage], then empty[slice][stage]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kModTmaSlices * kModTmaStages);
+  const int cols_per_block = (p.N6 + kModTmaCols - 1) / kModTmaCols;
+  const int blk = blockIdx.x / cols_per_block;
+  const int col_base = (blockIdx.x % cols_per_block) * kModTmaCols;
+  const int ncols = min(kModTmaCols, p.N6 - col_base);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool is_producer_warp = warp == kModTmaComputeThreads / 32;
+  const int cg = threadIdx.x % (kModTmaCols / 8);
+  const int slice = is_producer_warp ? lane : threadIdx.x / (kModTmaCols / 8);      // producer lane s serves slice s
+  const bool col_ok = cg * 8 < ncols;
+  const float* bias = p.b_ada0 + blk * p.b_block_stride;
+  const int c_per = (p.C + kModTmaSlices - 1) / kModTmaSlices;
+  const int c0 = min(p.C, slice * c_per), c1 = min(p.C, c0 + c_per);
+  const int n_groups = (is_producer_warp && lane >= kModTmaSlices) ? 0 : (c1 - c0 + kModTmaRows - 1) / kModTmaRows;
+  uint8_t* my_ring = ring + static_cast<size_t>(slice & (kModTmaSlices - 1)) * kModTmaStages * kModTmaRows * kModTmaCols * 2;
+  auto full_bar = [&](int st) { return smem_u32(bars + (slice & (kModTmaSlices - 1)) * kModTmaStages + st); };
+  auto empty_bar = [&](int st) { return smem_u32(bars + (kModTmaSlices + (slice & (kModTmaSlices - 1))) * kModTmaStages + st); };
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < kModTmaSlices * kModTmaStages; ++i) {
+      mbar_init(smem_u32(bars + i), 1);                                   // full: the producer's expect_tx arrival
+      mbar_init(smem_u32(bars + kModTmaSlices * kModTmaStages + i), 2);    // empty: the slice's two warps
+    }
+    fence_mbar_init();
+  }
+  int used = 0;                                // stage uses so far (keeps the barrier phases across request groups)
+  bool ok = true;
+  for (int r0 = 0; r0 < p.R; r0 += kModReqGroup) {
+    const int g = min(kModReqGroup, p.R - r0);
+    __syncthreads();                           // barriers exist; previous group's partials have been read
+    for (int i = threadIdx.x; i < kModReqGroup * p.C; i += kModTmaThreads) {
+      const int cc = i >> 3, rr = i & 7;
+      float v = 0.f;
+      if (rr < g) {
+        const float x = __bfloat162float(p.cond[static_cast<size_t>(r0 + rr) * p.C + cc]);
+        v = x / (1.0f + __expf(-x));
+      }
+      s_act[i] = v;
+    }
+    __syncthreads();
+    if (is_producer_warp) {
+      // ------------------------------------------------------------------ producer (lanes 0..3, one slice each)
+      for (int k = 0; k < n_groups && ok; ++k) {
+        const int u = used + k, st = u % kModTmaStages;
+        if (k >= kModTmaStages && !mbar_wait(empty_bar(st), ((u / kModTmaStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        const int r_first = c0 + k * kModTmaRows, n = min(kModTmaRows, c1 - r_first);
+        // two boxes of 256 columns x kModTmaRows rows (rows past C and columns past 6H arrive as zeros; rows that
+        // belong to the next slice are simply not used)
+        (void)n;
+        const int halves = ncols > 256 ? 2 : 1;
+        mbar_arrive_expect_tx(full_bar(st), static_cast<uint32_t>(halves) * kModTmaRows * 512u);
+        for (int hf = 0; hf < halves; ++hf)
+          tma_load_3d(smem_u32(my_ring + (static_cast<size_t>(st) * 2 + hf) * kModTmaRows * 512), &tmW, col_base + hf * 256, r_first, blk,
+                      full_bar(st));
+      }
+      used += n_groups;
+    } else {
+      // ------------------------------------------------------------------ compute warps
+      float2 acc[kModReqGroup][4];
+#pragma unroll
+      for (int rr = 0; rr < kModReqGroup; ++rr)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[rr][q] = make_float2(0.f, 0.f);
+      for (int k = 0; k < n_groups; ++k, ++used) {
+        const int st = used % kModTmaStages; const uint32_t ph = (used / kModTmaStages) & 1u;
+        if (ok && !__all_sync(0xffffffffu, mbar_wait(full_bar(st), ph, abort_flag))) ok = false;
+        if (ok && col_ok) {
+          const int r_first = c0 + k * kModTmaRows, n = min(kModTmaRows, c1 - r_first);
+          const uint8_t* rows = my_ring + (static_cast<size_t>(st) * 2 + (cg >> 5)) * kModTmaRows * 512 + (cg & 31) * 16;
+#pragma unroll
+          for (int j = 0; j < kModTmaRows; ++j) {
+            if (j < n) {
+              const uint4 raw = *reinterpret_cast<const uint4*>(rows + static_cast<size_t>(j) * 512);
+              const uint32_t u4[4] = {raw.x, raw.y, raw.z, raw.w};
+              float2 wf[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) wf[q] = make_float2(__uint_as_float(u4[q] << 16), __uint_as_float(u4[q] & 0xFFFF0000u));
+              const float4 a_lo = *reinterpret_cast<const float4*>(s_act + static_cast<size_t>(r_first + j) * 8);
+              const float4 a_hi = *reinterpret_cast<const float4*>(s_act + static_cast<size_t>(r_first + j) * 8 + 4);
+              const float a[8] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w, a_hi.x, a_hi.y, a_hi.z, a_hi.w};
+#pragma unroll
+              for (int rr = 0; rr < kModReqGroup; ++rr) {
+                const float2 aa = make_float2(a[rr], a[rr]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[rr][q] = ffma2(aa, wf[q], acc[rr][q]);
+              }
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(st));         // this warp is done with the stage
+      }
+      __syncwarp();
+      // the partials go into the activation buffer once every compute warp has finished with it (below)
+      asm volatile("bar.sync 1, %0;" ::"n"(kModTmaComputeThreads));
+#pragma unroll
+      for (int rr = 0; rr < kModReqGroup; ++rr)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          s_part[(slice * kModReqGroup + rr) * kModTmaCols + cg * 8 + 2 * q] = acc[rr][q].x;
+          s_part[(slice * kModReqGroup + rr) * kModTmaCols + cg * 8 + 2 * q + 1] = acc[rr][q].y;
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < g * kModTmaCols; i += kModTmaThreads) {
+      const int rr = i / kModTmaCols, cc = i % kModTmaCols;
+      if (col_base + cc < p.N6) {
+        float v = 0.f;
+#pragma unroll
+        for (int sl = 0; sl < kModTmaSlices; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModTmaCols + cc];
+        p.mod[(static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc] = v + bias[col_base + cc];
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicMax(status, kStatusModTimeout);
+}
+
+// ------------------------------------------------------------------------------------------------
 // LayerNorm (over H, biased variance, eps inside the root, no affine) + adaLN modulate:
 //   h[row, :] = (x - mean) * rstd * (1 + scale[req]) + shift[req]        -> fp16
 // One warp per row, the row held in registers (kVec float4 per lane: H <= 128 * kVec), two-pass
