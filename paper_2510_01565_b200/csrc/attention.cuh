@@ -86,16 +86,17 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  // ---- which (request, head, 256-row query block) this CTA owns
-  const int head = blockIdx.x % p.n_heads;
-  int qb = blockIdx.x / p.n_heads;
+  // ---- which (request, head, 256-row query block) this CTA owns: requests longest first, and within a
+  // request head-major, so that the CTAs resident at one time share the K/V of a few heads (a long
+  // request's K/V over all heads is larger than L2)
+  int head = 0, qb = blockIdx.x;
   int row_begin = 0, len = 0;
   for (int i = 0; i < seq.n; ++i) {
     const int r = seq.order[i];
     const int l = seq.cu[r + 1] - seq.cu[r];
     const int nb = (l + C::Q_ROWS - 1) / C::Q_ROWS;
-    if (qb < nb) { row_begin = seq.cu[r]; len = l; break; }
-    qb -= nb;
+    if (qb < nb * p.n_heads) { row_begin = seq.cu[r]; len = l; head = qb / nb; qb -= head * nb; break; }
+    qb -= nb * p.n_heads;
   }
   const int q_row0 = row_begin + qb * C::Q_ROWS;
   const int nkv = (len + 127) >> 7;
