@@ -66,7 +66,7 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = (BN / 2) * BK * 2;                  // this CTA's half of the weight tile
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
-constexpr int EPI_STAGE_FLOATS = 32 * 33;          // per epilogue warp: 32 rows x 32 columns, padded
+constexpr int EPI_STAGE_FLOATS = 32 * 36;          // per epilogue warp: 32 rows x 32 columns, rows padded to 144 bytes
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * EPI_STAGE_FLOATS * 4;
 }  // namespace gemm_cfg
 
@@ -76,6 +76,18 @@ __device__ __forceinline__ float gelu_tanh_f32(float z) {
   float t;
   asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(y));
   return 0.5f * z * (1.0f + t);
+}
+// The same function on two values with packed fp32 arithmetic (the epilogue shares its scheduler with
+// the MMA-issuing and the TMA-issuing warps: fewer instructions leave them more issue slots).
+__device__ __forceinline__ float2 gelu_tanh_f32x2(float2 z) {
+  const float k0 = 0.7978845608028654f, k1 = 0.044715f;
+  const float2 inner = ffma2(fmul2(z, z), make_float2(k0 * k1, k0 * k1), make_float2(k0, k0));
+  const float2 y = fmul2(inner, z);
+  float2 t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t.x) : "f"(y.x));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t.y) : "f"(y.y));
+  const float2 hz = fmul2(z, make_float2(0.5f, 0.5f));
+  return ffma2(hz, t, hz);
 }
 
 // Tile order.  Row tiles are grouped in bands of `band`; inside a band the row index runs fastest and
@@ -217,6 +229,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const float* gate = p.gate + ((DUAL && kind) ? p.gate_kind_stride : 0);
       const int req0 = __shfl_sync(0xffffffffu, my_req, 0);
       const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
+      // fp32 epilogues: this lane stores columns (lane % 8) * 4 .. + 3 of rows it * 4 + lane / 8, it < 8
+      int row_req[8];
+      unsigned store_rows = 0;
+      if (EPI == kEpiGateResidF32 || EPI == kEpiBiasF32) {
+#pragma unroll
+        for (int i8 = 0; i8 < 8; ++i8) {
+          const int rr = i8 * 4 + (lane >> 3);
+          row_req[i8] = __shfl_sync(0xffffffffu, my_req, rr);
+          const int rk = DUAL ? __shfl_sync(0xffffffffu, my_kind, rr) : 0;
+          if (m0 + quarter * 32 + rr < p.M && (!DUAL || rk == kind)) store_rows |= 1u << i8;
+        }
+      }
       // Residual rows of this tile do not depend on the accumulator: the first four 32-column chunks
       // are requested before waiting for the MMAs, later chunks four iterations ahead.
       const int cg = (lane & 7) * 4;
@@ -319,9 +343,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (EPI == kEpiGateResidF32 || EPI == kEpiBiasF32) {
           // Transpose through shared memory so that each global access covers whole 128-byte row
           // segments: lane -> (row it*4 + lane/8, columns (lane%8)*4 .. +3).
+          // Rows are padded to 36 floats: 16-byte accesses of both phases are free of bank conflicts.
           float* st = epi_stage + (warp - 2) * EPI_STAGE_FLOATS;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) st[lane * 33 + i] = __uint_as_float(r[i]);
+          for (int i = 0; i < 32; i += 4)
+            *reinterpret_cast<uint4*>(st + lane * 36 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
           __syncwarp();
           const int col = col0 + cg;                        // N is a multiple of 64: the whole chunk is inside
           {
@@ -338,19 +364,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int it = 0; it < 8; ++it) {
               const int rr = it * 4 + (lane >> 3);
               const int grow = m0 + quarter * 32 + rr;
-              const int rq = __shfl_sync(0xffffffffu, my_req, rr);
-              const int rk = DUAL ? __shfl_sync(0xffffffffu, my_kind, rr) : 0;
-              if (grow < p.M && (!DUAL || rk == kind)) {
-                if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(gate + rq * p.gate_stride + col));
-                const float* a = st + rr * 33 + cg;
+              if ((store_rows >> it) & 1u) {
+                if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(gate + row_req[it] * p.gate_stride + col));
+                const float4 a = *reinterpret_cast<const float4*>(st + rr * 36 + cg);
+                const float2 s0 = fadd2(make_float2(a.x, a.y), make_float2(b.x, b.y));
+                const float2 s1 = fadd2(make_float2(a.z, a.w), make_float2(b.z, b.w));
                 float4 o;
                 if (EPI == kEpiGateResidF32) {
-                  o.x = x[it].x + g.x * (a[0] + b.x);
-                  o.y = x[it].y + g.y * (a[1] + b.y);
-                  o.z = x[it].z + g.z * (a[2] + b.z);
-                  o.w = x[it].w + g.w * (a[3] + b.w);
+                  const float2 o0 = ffma2(make_float2(g.x, g.y), s0, make_float2(x[it].x, x[it].y));
+                  const float2 o1 = ffma2(make_float2(g.z, g.w), s1, make_float2(x[it].z, x[it].w));
+                  o = make_float4(o0.x, o0.y, o1.x, o1.y);
                 } else {
-                  o = make_float4(a[0] + b.x, a[1] + b.y, a[2] + b.z, a[3] + b.w);
+                  o = make_float4(s0.x, s0.y, s1.x, s1.y);
                 }
                 *reinterpret_cast<float4*>(p.out32 + static_cast<size_t>(grow) * p.N + col) = o;
               }
@@ -365,18 +390,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // bytes of each of 8 rows (whole sectors) instead of 16 bytes of each of 32 rows
             uint8_t* stb = reinterpret_cast<uint8_t*>(epi_stage + (warp - 2) * EPI_STAGE_FLOATS);
             uint4* srow = reinterpret_cast<uint4*>(stb + lane * 80);
+            const float4* bias4 = reinterpret_cast<const float4*>(bias + col0);   // col0 is a multiple of 32
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
               uint32_t w[4];
+              const float4 b0 = __ldg(bias4 + 2 * v), b1 = __ldg(bias4 + 2 * v + 1);
+              const float2 bb[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
                 const int i = 8 * v + 2 * h;
-                float a = __uint_as_float(r[i]), b = __uint_as_float(r[i + 1]);
-                if (FP8) { a *= sa * __ldg(p.col_scale + col0 + i); b *= sa * __ldg(p.col_scale + col0 + i + 1); }
-                a += __ldg(bias + col0 + i);
-                b += __ldg(bias + col0 + i + 1);
-                if (EPI == kEpiBiasGeluF16) { a = gelu_tanh_f32(a); b = gelu_tanh_f32(b); }
-                const __half2 hh = __floats2half2_rn(a, b);
+                float2 ab = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                if (FP8) { ab.x *= sa * __ldg(p.col_scale + col0 + i); ab.y *= sa * __ldg(p.col_scale + col0 + i + 1); }
+                ab = fadd2(ab, bb[h]);
+                if (EPI == kEpiBiasGeluF16) ab = gelu_tanh_f32x2(ab);
+                const __half2 hh = __floats2half2_rn(ab.x, ab.y);
                 w[h] = *reinterpret_cast<const uint32_t*>(&hh);
               }
               srow[v] = make_uint4(w[0], w[1], w[2], w[3]);
