@@ -194,8 +194,9 @@ dit_status dit_step_forward_requests(dit_ctx *ctx, const void *packed_tokens, co
 /* Same step with HOST buffers: copies tokens and cond to the device, runs the step, copies `out`
  * back, and returns after everything has drained (out is valid on return).  The transfers overlap the
  * step where the data flow allows it: the tokens go in as four row slices on a copy stream of the
- * context and block 0 normalises and projects each slice as it lands; the last GEMM runs in the same
- * row slices and every finished slice of `out` goes back while the next one computes.  The results are
+ * context and block 0 normalises and projects each slice as it lands; the part of the last block that
+ * follows attention runs in the same row slices (only its last GEMM for parallel blocks and in the
+ * e4m3 mode) and every finished slice of `out` goes back while the next one computes.  The results are
  * those of dit_step_forward bit for bit.  Use pinned host memory (pageable memory serialises the copies). */
 dit_status dit_step_forward_host(dit_ctx *ctx, const void *host_packed_tokens,
                                  const int32_t *per_request_token_lens, int32_t n_requests,

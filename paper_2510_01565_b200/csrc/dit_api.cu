@@ -301,7 +301,8 @@ cudaError_t launch_modulation(const ModParams& mp, int num_sms, size_t smem, cud
 }
 
 // `geo` (image geometry of the requests) is needed by the rotary term only; NULL otherwise.
-// `host_out` (dit_step_forward_host): the last GEMM runs in row slices and every finished slice of `out` is
+// `host_out` (dit_step_forward_host): the last block's row-wise part (everything after attention; for the
+// parallel form and the e4m3 mode only its last GEMM) runs in row slices and every finished slice of `out` is
 // copied to the host on the context's copy stream while the next slice computes.  `tokens_in_slices`: the
 // tokens are being copied in by the same slices (events tok_ready) and block 0 starts on each as it lands.
 dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int n, const void* cond, int n_blocks,
@@ -544,6 +545,52 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       } else {
         DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
       }
+      continue;
+    }
+    if (last && host_out && !dual && !fp8) {
+      // dit_step_forward_host, last block: after attention every row is independent, so projection, LayerNorm,
+      // up- and down-projection run slice by slice and a finished slice of the output goes to the host while
+      // the next one is computed.  A slice is a whole number of 256-row tiles: every element is computed
+      // exactly as in the unsliced launches.
+      const int tile_rows = 2 * gemm_cfg::BM;
+      const int per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;
+      for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
+        const int rows = std::min(per, T - r0);
+        const size_t eH = static_cast<size_t>(r0) * H, eF = static_cast<size_t>(r0) * F;
+        CUtensorMap tm_as, tm_hs, tm_us;
+        if (!make_map(ctx, &tm_as, a + eH, H, rows, gemm_cfg::BM) || !make_map(ctx, &tm_hs, h + eH, H, rows, gemm_cfg::BM) ||
+            !make_map(ctx, &tm_us, u + eF, F, rows, gemm_cfg::BM))
+          return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+        GemmParams q{};
+        q.status = status;
+        q.M = rows; q.row0 = r0; q.N = H; q.K = H;
+        q.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_o);
+        q.resid = stream + eH; q.out32 = stream + eH;
+        q.gate = modb + 2 * H; q.gate_stride = req_stride;
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_as, bs.tm_o, q, seq, st); }));
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
+          return launch_ln<false>(stream + eH, nullptr, h + eH, modb + 3 * H, modb + 4 * H, req_stride, rows, H, c.ln_eps, seq, st, ks, rg,
+                                  nullptr, ctx->num_sms, status, r0);
+        }));
+        q = GemmParams{};
+        q.status = status;
+        q.M = rows; q.row0 = r0; q.N = F; q.K = H;
+        q.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
+        q.out16 = u + eF;
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_hs, bs.tm_fc1, q, seq, st); }));
+        q = GemmParams{};
+        q.status = status;
+        q.M = rows; q.row0 = r0; q.N = H; q.K = F;
+        q.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
+        q.resid = stream + eH; q.out32 = out + eH;
+        q.gate = modb + 5 * H; q.gate_stride = req_stride;
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_us, bs.tm_fc2, q, seq, st); }));
+        DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->slice_done[sidx], st));
+        DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->slice_done[sidx], 0));
+        DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out + eH, out + eH, static_cast<size_t>(rows) * H * 4, cudaMemcpyDeviceToHost, ctx->copy_stream));
+      }
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, ctx->copy_stream));
+      ctx->host_copied = true;
       continue;
     }
     // output projection + gate + residual
