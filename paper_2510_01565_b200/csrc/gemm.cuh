@@ -280,11 +280,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             __syncwarp();                      // tcgen05.ld is warp-collective: reconverge first
             tmem_ld32(t_row + hc * HD + q * 32, r);
             tmem_ld_wait();
+            const float4* bias4 = reinterpret_cast<const float4*>(bias + colh + q * 32);   // colh is a multiple of HD
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              float acc_v = __uint_as_float(r[i]);
-              if (FP8) acc_v *= sa * __ldg(p.col_scale + colh + q * 32 + i);
-              v[q * 32 + i] = acc_v + __ldg(bias + colh + q * 32 + i);
+            for (int i = 0; i < 32; i += 4) {
+              const float4 b4 = __ldg(bias4 + (i >> 2));
+              float2 a0 = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+              float2 a1 = make_float2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+              if (FP8) {
+                const float4 cs = __ldg(reinterpret_cast<const float4*>(p.col_scale + colh + q * 32 + i));
+                a0 = fmul2(a0, make_float2(sa * cs.x, sa * cs.y));
+                a1 = fmul2(a1, make_float2(sa * cs.z, sa * cs.w));
+              }
+              a0 = fadd2(a0, make_float2(b4.x, b4.y));
+              a1 = fadd2(a1, make_float2(b4.z, b4.w));
+              v[q * 32 + i] = a0.x; v[q * 32 + i + 1] = a0.y; v[q * 32 + i + 2] = a1.x; v[q * 32 + i + 3] = a1.y;
             }
           }
           if (row_ok) {
@@ -292,12 +301,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (part < 2) {
               const float* g = (DUAL && kind) ? (part == 0 ? p.q_norm2 : p.k_norm2) : (part == 0 ? p.q_norm : p.k_norm);
               if (g) {
-                float ss = 0.f;
+                float2 ss2 = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int i = 0; i < HD; ++i) ss = fmaf(v[i], v[i], ss);
-                const float rstd = rsqrtf(ss * (1.0f / HD) + p.eps);
+                for (int i = 0; i < HD; i += 2) { const float2 t = make_float2(v[i], v[i + 1]); ss2 = ffma2(t, t, ss2); }
+                const float rstd = rsqrtf((ss2.x + ss2.y) * (1.0f / HD) + p.eps);
+                const float2 rs = make_float2(rstd, rstd);
 #pragma unroll
-                for (int i = 0; i < HD; ++i) v[i] *= rstd * __ldg(g + i);
+                for (int i = 0; i < HD; i += 4) {
+                  const float4 g4 = __ldg(reinterpret_cast<const float4*>(g + i));
+                  const float2 o0 = fmul2(make_float2(v[i], v[i + 1]), fmul2(rs, make_float2(g4.x, g4.y)));
+                  const float2 o1 = fmul2(make_float2(v[i + 2], v[i + 3]), fmul2(rs, make_float2(g4.z, g4.w)));
+                  v[i] = o0.x; v[i + 1] = o0.y; v[i + 2] = o1.x; v[i + 3] = o1.y;
+                }
               }
               if (p.rope_theta && (py | px)) {
                 constexpr int DT = HD / 8, NA = (HD - DT) / 2;   // unrotated channels, channels per axis group
