@@ -165,10 +165,17 @@ dit_status fail(dit_ctx* ctx, dit_status s, const char* fmt, const char* detail 
   return s;
 }
 
+// A failed CUDA call: the message holds the call's text (never used as a format string: it may contain
+// a '%') and the runtime's error string.
+dit_status fail_cuda(dit_ctx* ctx, const char* what, cudaError_t e) {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%.160s: %s", what, cudaGetErrorString(e));
+  return DIT_ERR_CUDA;
+}
+
 #define DIT_CUDA_TRY(ctx, expr)                                                        \
   do {                                                                                 \
     cudaError_t e_ = (expr);                                                           \
-    if (e_ != cudaSuccess) return fail(ctx, DIT_ERR_CUDA, #expr ": %s", cudaGetErrorString(e_)); \
+    if (e_ != cudaSuccess) return fail_cuda(ctx, #expr, e_);                           \
   } while (0)
 
 // 2-D fp16 tensor map: `inner` contiguous elements per row, `rows` rows, box 64 x box_rows, 128-byte swizzle,
