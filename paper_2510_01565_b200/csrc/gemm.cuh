@@ -452,7 +452,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);   // 8 arrivals: 4 warps x 2 CTAs
+      if (lane == 0) mbar_arrive_cluster_light(acc ? tempty_leader1 : tempty_leader0);   // 8 arrivals: 4 warps x 2 CTAs
     }
   }
 

@@ -241,6 +241,12 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same with the default (CTA-scope) release: no cluster-wide fence stalls the arriving warp.  Enough
+// where the arrival hands over tensor memory, whose accesses are ordered by tcgen05.wait and the
+// tcgen05 fences rather than by the memory model's scopes.
+__device__ __forceinline__ void mbar_arrive_cluster_light(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // TMA load issued by either CTA of a pair: data into the issuing CTA's shared memory, byte count
 // signalled on `bar_cluster`, a shared::cluster address (here: the leader CTA's barrier).  No multicast.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, int x, int y, uint32_t bar_cluster) {
