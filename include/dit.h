@@ -16,7 +16,10 @@
  *     memory.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Tokens, cond and weights cross the boundary as bf16; `out` is fp32.  Inside, GEMM operands
  *     are fp16 (bf16 weights ~N(0,0.02) convert exactly), accumulation, the residual stream and the
- *     modulation vectors are fp32.
+ *     modulation vectors are fp32.  Every narrowing store saturates: a value beyond fp16's range is
+ *     written as +-65504, never as infinity, so one request's overflow cannot become NaN in another
+ *     (masked attention probabilities are zeros multiplied by the neighbouring request's values).
+ *     DIT_FLAG_BF16_OPERANDS keeps bf16 operands instead.
  *   - The caller owns every buffer, including the workspace; the context owns only what it carves
  *     from the workspace.  No entry point below allocates device memory.
  *   - A context is not thread-safe; calls on one context must be issued serially (they may be
@@ -89,6 +92,14 @@ typedef struct {
  * the accumulator (fp32, exact products) is scaled back in the epilogue.  Everything else stays as
  * it is.  Errors grow to a few per cent of the output's rms; not available for two-stream blocks. */
 #define DIT_FLAG_FP8_GEMM 4u
+/* bf16 operands instead of fp16: the weights are kept as given (no conversion), the 16-bit
+ * activations (LayerNorm outputs, q/k/v, attention probabilities and output, GELU output) are stored
+ * as bf16, accumulation, residual stream and output stay fp32.  For checkpoints whose activations do
+ * not fit fp16's range (the fp16 path clamps such values to +-65504 instead of overflowing, see the
+ * Conventions above).  bf16 keeps 8 significant bits instead of 11, so the error against an exact
+ * evaluation is several times that of the fp16 path.  Plain sequential and parallel blocks only:
+ * the flag cannot be combined with the other three, and two-stream blocks are refused. */
+#define DIT_FLAG_BF16_OPERANDS 8u
 
 /* One request of the paper's problem statement (Section 3): an image resolution, a position in
  * its denoising schedule and the diffusion time of this step.  Image tokens = (height/16) *
@@ -213,6 +224,23 @@ typedef enum { DIT_TAP_H = 0, DIT_TAP_QKV = 1, DIT_TAP_ATTN = 2, DIT_TAP_U = 3, 
 dit_status dit_debug_tap(dit_ctx *ctx, dit_tap which, const void **ptr, int64_t *rows, int64_t *cols,
                          int32_t *elem_bytes);
 
+/* Test hooks that stand in for a memory checker.
+ * dit_debug_poison fills every activation region of the workspace (residual stream, h, qkv, a, u,
+ * modulation vectors, row scales, staging buffers, shell intermediates; not the weights) with 0xFF
+ * bytes, which read as NaN in every floating-point format used there, and writes a fixed pattern into
+ * the 1 KiB guard areas that follow the regions.  A step run afterwards turns any read of a row it
+ * never wrote into NaN in its output.  Asynchronous on `stream`.
+ * dit_debug_check_guards synchronises the device, compares the guard areas with the pattern and
+ * returns the number of damaged guards in *n_damaged (0 after any correct step). */
+dit_status dit_debug_poison(dit_ctx *ctx, void *stream);
+dit_status dit_debug_check_guards(dit_ctx *ctx, int32_t *n_damaged);
+
+/* Test hook for the failure path: launches one CTA that waits, with the library's bounded-wait
+ * routine and a limit of about 50 microseconds, on a barrier that nothing ever signals.  The wait runs
+ * out, the kernel returns normally and sets the device status word, so the next dit_ctx_poll_status
+ * returns DIT_ERR_TIMEOUT (once).  Nothing hangs or faults; the context stays usable. */
+dit_status dit_debug_expire_wait(dit_ctx *ctx, void *stream);
+
 /* Per-kernel timing for benchmarks.  While enabled, every kernel launch of a step is bracketed by
  * a pair of CUDA events on the step's stream (events are created on demand and kept; no device
  * memory is allocated).  dit_ctx_read_timing synchronises the device, adds up the elapsed time and
@@ -230,7 +258,9 @@ dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *laun
  * phase, a process whose memory pool belongs to a framework, a caller that was handed fixed buffers
  * and nothing else).  It needs no context and no workspace.
  *   mod_out[r, :] = W_ada^T SiLU(cond[r, :]) + b_ada        device [n_requests, 6H] fp32
- *   cond device [n_requests, C] bf16; w_ada device [C, 6H] bf16; b_ada device [6H] bf16 or NULL (zero)
+ *   cond device [n_requests, C] bf16; w_ada device [C, 6H] bf16, 16-byte aligned (it is read with
+ *   16-byte loads; DIT_ERR_INVALID_ARG otherwise, as for a mod_out that is not 4-byte aligned or a
+ *   cond / b_ada that is not 2-byte aligned); b_ada device [6H] bf16 or NULL (zero)
  * The result is that of the `mod` vectors dit_step_forward computes for that block (the same kernel; a
  * context with many blocks may sum the cond channels in wider groups, which moves the last fp32 bits).  The fp32 copy of
  * the bias, which the context path keeps in the caller's workspace, lives here in a fixed 96 KiB

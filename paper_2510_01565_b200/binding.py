@@ -19,6 +19,7 @@ DIT_OK = 0
 DIT_FLAG_QK_RMSNORM = 1
 DIT_FLAG_ROPE_2D = 2
 DIT_FLAG_FP8_GEMM = 4
+DIT_FLAG_BF16_OPERANDS = 8
 STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
                 "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
 KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
@@ -26,7 +27,7 @@ TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights", "dit_load_dual_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
-           "dit_ctx_poll_status", "dit_debug_tap", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_debug_poison", "dit_debug_check_guards", "dit_debug_expire_wait", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
            "dit_denoise_step", "dit_denoise_round", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
@@ -114,6 +115,12 @@ def load_library() -> C.CDLL:
     lib.dit_ctx_poll_status.argtypes = [vp]
     lib.dit_debug_tap.restype = C.c_int
     lib.dit_debug_tap.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+    lib.dit_debug_poison.restype = C.c_int
+    lib.dit_debug_poison.argtypes = [vp, vp]
+    lib.dit_debug_check_guards.restype = C.c_int
+    lib.dit_debug_check_guards.argtypes = [vp, C.POINTER(i32)]
+    lib.dit_debug_expire_wait.restype = C.c_int
+    lib.dit_debug_expire_wait.argtypes = [vp, vp]
     lib.dit_ctx_set_timing.restype = C.c_int
     lib.dit_ctx_set_timing.argtypes = [vp, i32]
     lib.dit_ctx_read_timing.restype = C.c_int
@@ -473,6 +480,20 @@ class DitContext:
     def dit_ctx_poll_status(self):
         self._check(self.lib.dit_ctx_poll_status(self.handle))
 
+    def dit_debug_poison(self, stream=None):
+        """Fills the activation regions of the workspace with NaN bytes and rewrites the guard areas."""
+        self._check(self.lib.dit_debug_poison(self.handle, self._stream(stream)))
+
+    def dit_debug_check_guards(self) -> int:
+        """Number of damaged guard areas (0 after a correct step)."""
+        n = C.c_int32(-1)
+        self._check(self.lib.dit_debug_check_guards(self.handle, C.byref(n)))
+        return int(n.value)
+
+    def dit_debug_expire_wait(self, stream=None):
+        """Launches the one-CTA kernel whose bounded wait runs out (sets the status word)."""
+        self._check(self.lib.dit_debug_expire_wait(self.handle, self._stream(stream)))
+
     def dit_ctx_set_timing(self, enabled: bool):
         self._check(self.lib.dit_ctx_set_timing(self.handle, 1 if enabled else 0))
 
@@ -486,11 +507,12 @@ class DitContext:
         return int(self.lib.dit_last_launch_count(self.handle))
 
     def dit_debug_tap(self, which: str):
-        """Copy of an internal buffer of the last step as a torch tensor (fp16 or fp32)."""
+        """Copy of an internal buffer of the last step as a torch tensor (fp16, bf16 in the bf16-operand mode, or fp32)."""
         torch = self.torch
         ptr, rows, cols, eb = C.c_void_p(), C.c_int64(), C.c_int64(), C.c_int32()
         self._check(self.lib.dit_debug_tap(self.handle, TAPS[which], C.byref(ptr), C.byref(rows), C.byref(cols), C.byref(eb)))
-        dtype = torch.float16 if eb.value == 2 else torch.float32
+        dtype16 = torch.bfloat16 if (self.cfg.flags & DIT_FLAG_BF16_OPERANDS) else torch.float16
+        dtype = dtype16 if eb.value == 2 else torch.float32
         base = (self.workspace.data_ptr() + 1023) // 1024 * 1024
         off = ptr.value - base
         torch.cuda.synchronize()

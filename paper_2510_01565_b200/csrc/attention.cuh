@@ -61,7 +61,8 @@ __device__ __forceinline__ float exp2_approx(float x) {
   return y;
 }
 
-template <int D>
+// BF16: q, k, v, P and the output are bf16 instead of fp16 (bf16-operand mode).
+template <int D, bool BF16 = false>
 __global__ void __launch_bounds__(AttnCfg<D>::THREADS, 1)
 attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnParams p,
                          const __grid_constant__ SeqInfo seq) {
@@ -151,7 +152,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       // A use waits for its K tile (first query tile) and for the warpgroup of use u - 1 to have read
       // the buffer out; the K stage is released after the last query tile.  This thread and the P V
       // issuer wait independently, so neither hand-off keeps the other's MMAs off the tensor pipe.
-      constexpr uint32_t idesc_s = idesc_f16(128, 128, false);
+      constexpr uint32_t idesc_s = idesc_f16(128, 128, false, BF16);
       const int ntile = tile1_valid ? 2 : 1;
       static_assert(C::KV_STAGES == 2, "descriptor selection below assumes two stages");
       const uint64_t qdesc0 = smem_desc_sw128(base + C::OFF_Q, 16, 1024);
@@ -176,7 +177,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       }
     } else if (warp == 2 && lane == 0) {
       // ------------------------------------------------------------------ MMA issuer 2: P V
-      constexpr uint32_t idesc_pv = idesc_f16(128, D, true);
+      constexpr uint32_t idesc_pv = idesc_f16(128, D, true, BF16);
       const int ntile = tile1_valid ? 2 : 1;
       // V: MN-major B.  16 keys = two 8-row groups (stride 1024 B); the next 64 head columns live
       // one panel further (leading byte offset).
@@ -276,8 +277,7 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
         const float2 x = ffma2(make_float2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2);
         const float2 e = make_float2(exp2_approx(x.x), exp2_approx(x.y));
         if (i & 2) rs1 = fadd2(rs1, e); else rs0 = fadd2(rs0, e);
-        const __half2 hh = __floats2half2_rn(e.x, e.y);
-        sv[i >> 1] = *reinterpret_cast<const uint32_t*>(&hh);
+        sv[i >> 1] = pack16x2<BF16>(e.x, e.y);
       }
       // P[tile] is still being read by the previous key block's P V until that product has finished;
       // by now (a whole tile of exponentials later) it normally has
@@ -297,7 +297,11 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       // the last P V product has landed: normalise and write this row
       if (!__all_sync(0xffffffffu, mbar_wait(o_full(tile), (nkv - 1) & 1u, abort_flag))) goto done;
       tc_fence_after();
-      const float inv = 1.0f / l;
+      // Far outside any sane range (|score * scale| beyond 2^24 or so, i.e. operands that were clamped
+      // at the edge of the 16-bit format) the fused multiply-add of the exponent no longer cancels the
+      // reference exactly and a row's probabilities can all underflow or overflow: such a row is written
+      // as zeros, never as NaN or infinity
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
       const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
       __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.ld_out + head * D;
 #pragma unroll 1
@@ -313,8 +317,10 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
               const int i = 8 * v + 2 * h;
-              const __half2 hh = __floats2half2_rn(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-              w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+              float o0 = __uint_as_float(r[i]) * inv, o1 = __uint_as_float(r[i + 1]) * inv;
+              if (!(fabsf(o0) <= 3.0e38f)) o0 = 0.f;
+              if (!(fabsf(o1) <= 3.0e38f)) o1 = 0.f;
+              w[h] = pack16x2<BF16>(o0, o1);
             }
             *(reinterpret_cast<uint4*>(dst + ch * 32) + v) = make_uint4(w[0], w[1], w[2], w[3]);
           }

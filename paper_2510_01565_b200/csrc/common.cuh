@@ -30,7 +30,7 @@ struct RowGeom {
 };
 
 // Device status word values (written by a kernel whose bounded wait ran out).
-enum : int { kStatusOk = 0, kStatusGemmTimeout = 1, kStatusAttnTimeout = 2, kStatusLnTimeout = 3, kStatusModTimeout = 4 };
+enum : int { kStatusOk = 0, kStatusGemmTimeout = 1, kStatusAttnTimeout = 2, kStatusLnTimeout = 3, kStatusModTimeout = 4, kStatusTestTimeout = 5 };
 
 // Request that owns packed row `row` (binary search over at most 64 entries).
 __device__ __forceinline__ int find_request(const SeqInfo& s, int row) {

@@ -42,8 +42,17 @@ struct Layout {
   size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
   size_t row_scale;    // per-row scales of the e4m3 activations (DIT_FLAG_FP8_GEMM)
   size_t items;        // two-stream launches: [0] item count, then per-tile flags, then the items
+  // test hooks: 1 KiB guard areas after the activation regions, and the [begin, end) ranges that
+  // dit_debug_poison fills
+  static constexpr int kMaxGuards = 16;
+  size_t guard[kMaxGuards];
+  int n_guards;
+  size_t poison_begin[kMaxGuards], poison_end[kMaxGuards];
+  int n_poison;
   size_t bytes;
 };
+constexpr size_t kGuardBytes = 1024;
+constexpr uint32_t kGuardPattern = 0xC3A55A3Cu;
 constexpr int kWoutRows = 256;   // W_out^T is stored zero-padded to one full weight tile of the GEMM
 
 bool config_ok(const dit_config* c) {
@@ -55,7 +64,9 @@ bool config_ok(const dit_config* c) {
   if (c->cond_dim < 1 || c->cond_dim > kMaxCondDim) return false;
   if (c->max_blocks < 1 || c->max_total_tokens < 1) return false;
   if (c->max_requests < 1 || c->max_requests > DIT_MAX_REQUESTS) return false;
-  if (!(c->ln_eps >= 0.f) || (c->flags & ~static_cast<uint32_t>(DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D | DIT_FLAG_FP8_GEMM))) return false;
+  if (!(c->ln_eps >= 0.f) || (c->flags & ~static_cast<uint32_t>(DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D | DIT_FLAG_FP8_GEMM | DIT_FLAG_BF16_OPERANDS))) return false;
+  // the bf16-operand mode is built for the plain sequential and parallel blocks only
+  if ((c->flags & DIT_FLAG_BF16_OPERANDS) && (c->flags & (DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D | DIT_FLAG_FP8_GEMM))) return false;
   return true;
 }
 
@@ -82,17 +93,30 @@ Layout make_layout(const dit_config& c) {
   L.blk.s_fc1 = take(F * 4);
   L.blk.bytes = o;
   o = 0;
+  // every activation region (or run of regions) is followed by a guard area and is listed as a poison range
+  auto guard = [&](size_t begin) {
+    L.poison_begin[L.n_poison] = begin; L.poison_end[L.n_poison++] = o;
+    L.guard[L.n_guards++] = take(kGuardBytes);
+  };
   L.weights = take(L.blk.bytes * c.max_blocks);
   L.stream = take(T * H * 4);
+  guard(L.stream);
   L.h = take(T * H * 2);
+  guard(L.h);
   L.qkv = take(T * 3 * H * 2);
-  L.a = take(T * H * 2);
+  guard(L.qkv);
+  L.a = take(T * H * 2);             // a and u stay neighbours: a parallel block uses them as one [T, H + F] buffer
   L.u = take(T * F * 2);
+  guard(L.a);
   L.mod = take(R * c.max_blocks * 6 * H * 4);
+  guard(L.mod);
   L.status = take(256);
   L.stage_tokens = take(T * H * 2);
+  guard(L.stage_tokens);
   L.stage_cond = take(R * C * 2);
+  guard(L.stage_cond);
   L.stage_out = take(T * H * 4);
+  guard(L.stage_out);
   L.sh_w_in = take(DIT_PATCH_DIM * H * 2);
   L.sh_b_in = take(H * 4);
   L.sh_w_t1 = take(DIT_T_EMB_DIM * C * 2);
@@ -109,8 +133,10 @@ Layout make_layout(const dit_config& c) {
   L.sh_modfin = take(R * 2 * H * 4);
   L.sh_vtok = take(T * DIT_PATCH_DIM * 4);
   L.sh_pooled = take(R * C * 4);
+  guard(L.sh_temb);
   L.rope_theta = take(64 * 4);
   L.row_scale = take(T * 4);
+  guard(L.row_scale);
   L.items = take((16 + 3 * (T / (2 * 128) + 2)) * 4);
   L.bytes = o;
   return L;
@@ -218,7 +244,7 @@ bool build_seq(const int32_t* lens, int n, SeqInfo* s) {
 
 const RowGeom kNoGeom{};
 
-template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false>
+template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false, bool BF16 = false>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                         const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom, const CUtensorMap* tmB2 = nullptr) {
   // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
@@ -228,15 +254,16 @@ cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtens
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);   // a two-stream launch may have more items than row tiles: the loop covers them
-  gemm_tcgen05_kernel<EPI, HD, DUAL, FP8><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
+  q.operand_bf16 = (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS) ? 1 : 0;
+  gemm_tcgen05_kernel<EPI, HD, DUAL, FP8, BF16><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
   return cudaGetLastError();
 }
 
-template <int D>
+template <int D, bool BF16 = false>
 cudaError_t launch_attention(const CUtensorMap& tmQKV, const AttnParams& p, const SeqInfo& seq, cudaStream_t st) {
   int qblocks = 0;
   for (int r = 0; r < seq.n; ++r) qblocks += (seq.cu[r + 1] - seq.cu[r] + AttnCfg<D>::Q_ROWS - 1) / AttnCfg<D>::Q_ROWS;
-  attention_tcgen05_kernel<D><<<qblocks * p.n_heads, AttnCfg<D>::THREADS, AttnCfg<D>::SMEM_BYTES, st>>>(tmQKV, p, seq);
+  attention_tcgen05_kernel<D, BF16><<<qblocks * p.n_heads, AttnCfg<D>::THREADS, AttnCfg<D>::SMEM_BYTES, st>>>(tmQKV, p, seq);
   return cudaGetLastError();
 }
 
@@ -261,22 +288,23 @@ template <bool kFromBf16, bool kOutFp8 = false>
 cudaError_t launch_ln(const void* xin, float* stream_out, __half* h, const float* shift0, const float* scale0,
                       long long req_stride, int T, int H, float eps, const SeqInfo& seq, cudaStream_t st,
                       long long kind_stride = 0, const RowGeom& geo = kNoGeom, float* row_scale = nullptr,
-                      int num_sms = 0, int* status = nullptr, int row0 = 0) {
+                      int num_sms = 0, int* status = nullptr, int row0 = 0, bool out_bf16 = false) {
   const bool cache_vectors = kind_stride == 0;
+  const int ob = out_bf16 ? 1 : 0;
   const int slots = ln_tma_slots(H, kFromBf16, cache_vectors);
   if (num_sms > 0 && status && slots >= 1 && T >= 4 * num_sms) {
     const int grid = std::min(num_sms, (T + kLnTmaWarps - 1) / kLnTmaWarps), block = kLnTmaWarps * 32;
     const size_t smem = ln_tma_smem(H, kFromBf16, cache_vectors, slots);
     const int cv = cache_vectors ? 1 : 0;
-    if (H <= 1024) ln_modulate_tma_kernel<kFromBf16, 8, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
-    else if (H <= 3072) ln_modulate_tma_kernel<kFromBf16, 24, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
-    else ln_modulate_tma_kernel<kFromBf16, 32, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0);
+    if (H <= 1024) ln_modulate_tma_kernel<kFromBf16, 8, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0, ob);
+    else if (H <= 3072) ln_modulate_tma_kernel<kFromBf16, 24, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0, ob);
+    else ln_modulate_tma_kernel<kFromBf16, 32, kOutFp8><<<grid, block, smem, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, slots, cv, status, row0, ob);
     return cudaGetLastError();
   }
   const int grid = (T + kLnWarps - 1) / kLnWarps, block = kLnWarps * 32;
-  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
-  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
-  else ln_modulate_kernel<kFromBf16, 32, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0);
+  if (H <= 1024) ln_modulate_kernel<kFromBf16, 8, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0, ob);
+  else if (H <= 3072) ln_modulate_kernel<kFromBf16, 24, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0, ob);
+  else ln_modulate_kernel<kFromBf16, 32, kOutFp8><<<grid, block, 0, st>>>(xin, stream_out, h, shift0, scale0, req_stride, T, H, eps, seq, kind_stride, geo, row_scale, row0, ob);
   return cudaGetLastError();
 }
 
@@ -320,6 +348,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   if (!build_seq(lens, n, &seq)) return fail(ctx, DIT_ERR_INVALID_ARG, "every request needs at least one token");
   const bool qk_variant = (c.flags & (DIT_FLAG_QK_RMSNORM | DIT_FLAG_ROPE_2D)) != 0;
   const bool fp8 = (c.flags & DIT_FLAG_FP8_GEMM) != 0;     // QKV and up-projection read e4m3 h and weights
+  const bool bf = (c.flags & DIT_FLAG_BF16_OPERANDS) != 0; // h, qkv, a, u and the weights are bf16 instead of fp16
   if ((c.flags & DIT_FLAG_ROPE_2D) && !geo)
     return fail(ctx, DIT_ERR_INVALID_ARG, "the rotary term needs the requests' geometry: use dit_step_forward_requests");
   const int T = seq.total, H = c.hidden, F = c.mlp_hidden;
@@ -474,8 +503,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
           return b == 0 ? launch_ln<true, true>(tokens, stream, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
                         : launch_ln<false, true>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status);
         return b == 0 ? launch_ln<true>(static_cast<const __nv_bfloat16*>(tokens) + e0, stream + e0, h + e0, modb, modb + H, req_stride, rows, H,
-                                        c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status, r0)
-                      : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
+                                        c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status, r0, bf)
+                      : launch_ln<false>(stream, nullptr, h, modb, modb + H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status, 0, bf);
       }));
       GemmParams q = g;
       q.M = rows; q.row0 = r0; q.out16 = qkv + static_cast<size_t>(r0) * 3 * H;
@@ -493,6 +522,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       } else {
         DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_QKV, [&] {
           if (fp8) return launch_gemm<kEpiBiasF16, 0, false, true>(ctx, tmA, bs.tm_qkv, q, seq, st);
+          if (bf) return launch_gemm<kEpiBiasF16, 0, false, false, true>(ctx, tmA, bs.tm_qkv, q, seq, st);
           return dual ? launch_gemm<kEpiBiasF16, 0, true>(ctx, tmA, bs.tm_qkv, q, seq, st, rg, &bt.tm_qkv)
                       : launch_gemm<kEpiBiasF16>(ctx, tmA, bs.tm_qkv, q, seq, st);
         }));
@@ -525,6 +555,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
     ap.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c.head_dim));
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_ATTENTION, [&] {
+      if (bf) return c.head_dim == 128 ? launch_attention<128, true>(tm_qkv, ap, seq, st) : launch_attention<64, true>(tm_qkv, ap, seq, st);
       return c.head_dim == 128 ? launch_attention<128>(tm_qkv, ap, seq, st) : launch_attention<64>(tm_qkv, ap, seq, st);
     }));
     if (bs.parallel) {
@@ -536,6 +567,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       g.out16 = cat + H; g.ld16 = H + F;
       if (fp8) { g.row_scale = row_scale; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc1); }
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
+        if (bf) return launch_gemm<kEpiBiasGeluF16, 0, false, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st);
         return fp8 ? launch_gemm<kEpiBiasGeluF16, 0, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st)
                    : launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st);
       }));
@@ -577,14 +609,17 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
         DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_as, bs.tm_o, q, seq, st); }));
         DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
           return launch_ln<false>(stream + eH, nullptr, h + eH, modb + 3 * H, modb + 4 * H, req_stride, rows, H, c.ln_eps, seq, st, ks, rg,
-                                  nullptr, ctx->num_sms, status, r0);
+                                  nullptr, ctx->num_sms, status, r0, bf);
         }));
         q = GemmParams{};
         q.status = status;
         q.M = rows; q.row0 = r0; q.N = F; q.K = H;
         q.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc1);
         q.out16 = u + eF;
-        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] { return launch_gemm<kEpiBiasGeluF16>(ctx, tm_hs, bs.tm_fc1, q, seq, st); }));
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
+          return bf ? launch_gemm<kEpiBiasGeluF16, 0, false, false, true>(ctx, tm_hs, bs.tm_fc1, q, seq, st)
+                    : launch_gemm<kEpiBiasGeluF16>(ctx, tm_hs, bs.tm_fc1, q, seq, st);
+        }));
         q = GemmParams{};
         q.status = status;
         q.M = rows; q.row0 = r0; q.N = H; q.K = F;
@@ -615,7 +650,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     // LN2 + modulate
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_LN_MODULATE, [&] {
       return fp8 ? launch_ln<false, true>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, row_scale, ctx->num_sms, status)
-                 : launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status);
+                 : launch_ln<false>(stream, nullptr, h, modb + 3 * H, modb + 4 * H, req_stride, T, H, c.ln_eps, seq, st, ks, rg, nullptr, ctx->num_sms, status, 0, bf);
     }));
     // MLP up-projection + GELU-tanh
     g = GemmParams{};
@@ -627,6 +662,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     if (fp8) { g.row_scale = row_scale; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc1); }
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC1, [&] {
       if (fp8) return launch_gemm<kEpiBiasGeluF16, 0, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st);
+      if (bf) return launch_gemm<kEpiBiasGeluF16, 0, false, false, true>(ctx, tm_h, bs.tm_fc1, g, seq, st);
       return dual ? launch_gemm<kEpiBiasGeluF16, 0, true>(ctx, tm_h, bs.tm_fc1, g, seq, st, rg, &bt.tm_fc1)
                   : launch_gemm<kEpiBiasGeluF16>(ctx, tm_h, bs.tm_fc1, g, seq, st);
     }));
@@ -751,6 +787,10 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16, 0, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16, 0, false, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16, 0, false, false, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128, true>), AttnCfg<128>::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64, true>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<128>), AttnCfg<128>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&attention_tcgen05_kernel<64>), AttnCfg<64>::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu>), mod_smem_bytes(kMaxCondDim));  // same for every context
@@ -796,6 +836,10 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->tok_ready[i], cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->copies_done, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
+  for (int g = 0; g < lay.n_guards && e == cudaSuccess; ++g) {
+    fill_u32_kernel<<<1, 256>>>(reinterpret_cast<uint32_t*>(ctx->ws + lay.guard[g]), kGuardPattern, static_cast<int>(kGuardBytes / 4));
+    e = cudaGetLastError();
+  }
   if (e == cudaSuccess) {
     // rotary pair frequencies of one axis group of n = (d - d/8) / 2 channels: 10000^(-2i/n), i < n/2
     float theta[64] = {};
@@ -842,7 +886,10 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   };
   auto weight = [&](const void* src, size_t off, int K, int N) {   // [K, N] bf16 -> [N, K] fp16
     dim3 grid((N + 31) / 32, (K + 31) / 32);
-    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    if (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS)
+      transpose_bf16_to_f16_kernel<true><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    else
+      transpose_bf16_to_f16_kernel<false><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
     return cudaGetLastError();
   };
   const bool fp8 = (ctx->cfg.flags & DIT_FLAG_FP8_GEMM) != 0;
@@ -879,6 +926,7 @@ dit_status dit_load_dual_block_weights(dit_ctx* ctx, int32_t b, const dit_block_
   ctx->err[0] = 0;
   if (b < 0 || b + 1 >= ctx->cfg.max_blocks) return fail(ctx, DIT_ERR_CAPACITY, "a two-stream block needs slots b and b + 1 inside [0, max_blocks)");
   if (ctx->cfg.flags & DIT_FLAG_FP8_GEMM) return fail(ctx, DIT_ERR_SHAPE, "two-stream blocks are not available with DIT_FLAG_FP8_GEMM");
+  if (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS) return fail(ctx, DIT_ERR_SHAPE, "two-stream blocks are not available with DIT_FLAG_BF16_OPERANDS");
   dit_status s = dit_load_block_weights(ctx, b, image_stream, stream);
   if (s != DIT_OK) return s;
   s = dit_load_block_weights(ctx, b + 1, text_stream, stream);
@@ -914,7 +962,10 @@ dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_pa
   };
   auto weight = [&](const void* src, size_t off, int K, int N) {   // [K, N] bf16 -> [N, K] fp16
     dim3 grid((N + 31) / 32, (K + 31) / 32);
-    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    if (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS)
+      transpose_bf16_to_f16_kernel<true><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
+    else
+      transpose_bf16_to_f16_kernel<false><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), reinterpret_cast<__half*>(base + off), K, N);
     return cudaGetLastError();
   };
   DIT_CUDA_TRY(ctx, cudaMemsetAsync(base + L.b_ada, 0, static_cast<size_t>(6) * H * 4, st));
@@ -1047,7 +1098,8 @@ dit_status dit_ctx_poll_status(dit_ctx* ctx) {
   if (word[0] == kStatusOk) return DIT_OK;
   DIT_CUDA_TRY(ctx, cudaMemset(ctx->ws + ctx->lay.status, 0, sizeof(word)));
   return fail(ctx, DIT_ERR_TIMEOUT, "a bounded wait ran out in the %s kernel",
-              word[0] == kStatusGemmTimeout ? "GEMM" : (word[0] == kStatusAttnTimeout ? "attention" : (word[0] == kStatusLnTimeout ? "LayerNorm" : "modulation")));
+              word[0] == kStatusGemmTimeout ? "GEMM" : (word[0] == kStatusAttnTimeout ? "attention" : (word[0] == kStatusLnTimeout ? "LayerNorm" :
+              (word[0] == kStatusTestTimeout ? "wait-expiry test" : "modulation"))));
 }
 
 dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t* rows, int64_t* cols, int32_t* elem_bytes) {
@@ -1064,6 +1116,42 @@ dit_status dit_debug_tap(dit_ctx* ctx, dit_tap which, const void** ptr, int64_t*
     case DIT_TAP_STREAM: *ptr = ctx->ws + ctx->lay.stream; *rows = T; *cols = H; *elem_bytes = 4; break;
     default: return DIT_ERR_INVALID_ARG;
   }
+  return DIT_OK;
+}
+
+dit_status dit_debug_poison(dit_ctx* ctx, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = ctx->lay;
+  for (int i = 0; i < L.n_poison; ++i)
+    DIT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->ws + L.poison_begin[i], 0xFF, L.poison_end[i] - L.poison_begin[i], st));
+  for (int g = 0; g < L.n_guards; ++g) {
+    fill_u32_kernel<<<1, 256, 0, st>>>(reinterpret_cast<uint32_t*>(ctx->ws + L.guard[g]), kGuardPattern, static_cast<int>(kGuardBytes / 4));
+    DIT_CUDA_TRY(ctx, cudaGetLastError());
+  }
+  return DIT_OK;
+}
+
+dit_status dit_debug_check_guards(dit_ctx* ctx, int32_t* n_damaged) {
+  if (!ctx || !n_damaged) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  *n_damaged = 0;
+  DIT_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  uint32_t host[kGuardBytes / 4];
+  for (int g = 0; g < ctx->lay.n_guards; ++g) {
+    DIT_CUDA_TRY(ctx, cudaMemcpy(host, ctx->ws + ctx->lay.guard[g], kGuardBytes, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < kGuardBytes / 4; ++i)
+      if (host[i] != kGuardPattern) { ++*n_damaged; break; }
+  }
+  return DIT_OK;
+}
+
+dit_status dit_debug_expire_wait(dit_ctx* ctx, void* stream) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->at<int>(ctx->lay.status));
+  DIT_CUDA_TRY(ctx, cudaGetLastError());
   return DIT_OK;
 }
 
@@ -1198,7 +1286,8 @@ dit_status final_impl(dit_ctx* ctx, const float* x, const SeqInfo& seq, const Sh
   if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM)) return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   DIT_CUDA_TRY(ctx, launch_small_linear<kModInCondSilu>(cond, ctx->ws + ctx->lay.sh_w_fa, ctx->at<float>(ctx->lay.sh_b_fa), nullptr,
                                                         modfin, nullptr, n, c.cond_dim, 2 * H, st));
-  DIT_CUDA_TRY(ctx, launch_ln<false>(x, nullptr, h, modfin, modfin + H, 2ll * H, T, H, c.ln_eps, seq, st, 0, kNoGeom, nullptr, ctx->num_sms, ctx->at<int>(ctx->lay.status)));
+  DIT_CUDA_TRY(ctx, launch_ln<false>(x, nullptr, h, modfin, modfin + H, 2ll * H, T, H, c.ln_eps, seq, st, 0, kNoGeom, nullptr, ctx->num_sms, ctx->at<int>(ctx->lay.status),
+                                     0, (c.flags & DIT_FLAG_BF16_OPERANDS) != 0));
   GemmParams g{};
   g.status = ctx->at<int>(ctx->lay.status);
   g.M = T; g.N = DIT_PATCH_DIM; g.K = H;
@@ -1255,8 +1344,12 @@ dit_status dit_load_shell_weights(dit_ctx* ctx, const dit_shell_weights* w, void
   DIT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->ws + L.sh_w_out, 0, kWoutRows * H * 2, st));
   {
     dim3 grid((DIT_PATCH_DIM + 31) / 32, static_cast<unsigned>((H + 31) / 32));
-    transpose_bf16_to_f16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w->w_out), ctx->at<__half>(L.sh_w_out),
-                                                       static_cast<int>(H), DIT_PATCH_DIM);
+    if (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS)
+      transpose_bf16_to_f16_kernel<true><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w->w_out), ctx->at<__half>(L.sh_w_out),
+                                                               static_cast<int>(H), DIT_PATCH_DIM);
+    else
+      transpose_bf16_to_f16_kernel<false><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w->w_out), ctx->at<__half>(L.sh_w_out),
+                                                                static_cast<int>(H), DIT_PATCH_DIM);
     DIT_CUDA_TRY(ctx, cudaGetLastError());
   }
   if (!make_map(ctx, &ctx->tm_wout, ctx->ws + L.sh_w_out, H, kWoutRows, gemm_cfg::BN / 2))
@@ -1491,6 +1584,10 @@ extern "C" dit_status dit_modulation_noalloc(const void* cond, const void* w_ada
   if (n_requests < 0) return DIT_ERR_INVALID_ARG;
   if (n_requests == 0) return DIT_OK;
   if (!cond || !w_ada || !mod_out) return DIT_ERR_INVALID_ARG;
+  // W_ada is read with 16-byte loads (rows are 6H bf16 = a multiple of 16 bytes, so the base decides)
+  if (reinterpret_cast<uintptr_t>(w_ada) % 16 || reinterpret_cast<uintptr_t>(mod_out) % 4 ||
+      reinterpret_cast<uintptr_t>(cond) % 2 || reinterpret_cast<uintptr_t>(b_ada) % 2)
+    return DIT_ERR_INVALID_ARG;
   if (hidden < 64 || hidden % 64 || cond_dim < 1) return DIT_ERR_SHAPE;
   if (hidden > kNoAllocMaxHidden || cond_dim > kNoAllocMaxCond || n_requests > DIT_MAX_REQUESTS) return DIT_ERR_CAPACITY;
   float* scratch = nullptr;

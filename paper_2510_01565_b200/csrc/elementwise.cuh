@@ -282,7 +282,7 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
 
 // ------------------------------------------------------------------------------------------------
 // LayerNorm (over H, biased variance, eps inside the root, no affine) + adaLN modulate:
-//   h[row, :] = (x - mean) * rstd * (1 + scale[req]) + shift[req]        -> fp16
+//   h[row, :] = (x - mean) * rstd * (1 + scale[req]) + shift[req]        -> fp16 (bf16 with out_bf16)
 // One warp per row, the row held in registers (kVec float4 per lane: H <= 128 * kVec), two-pass
 // statistics, fixed shuffle order.  Small CTAs (4 rows) and a register budget that lets several CTAs
 // share an SM keep enough loads in flight to cover HBM latency.
@@ -297,7 +297,7 @@ constexpr int kLnWarps = 4;
 template <bool kFromBf16, int kLnMaxVec, bool kOutFp8>
 __device__ __forceinline__ void ln_modulate_row(const void* src, int row, int lane, float* __restrict__ stream_out,
                                                 __half* __restrict__ h, const float4* sh, const float4* sc, int H,
-                                                float eps, float* __restrict__ row_scale) {
+                                                float eps, float* __restrict__ row_scale, bool out_bf16) {
   const int nvec = H >> 2;
   float4 v[kLnMaxVec];
   float sum = 0.f;
@@ -370,8 +370,8 @@ __device__ __forceinline__ void ln_modulate_row(const void* src, int row, int la
       const float b = (v[i].y - mean) * rstd * (1.f + s1.y) + s0.y;
       const float c = (v[i].z - mean) * rstd * (1.f + s1.z) + s0.z;
       const float d = (v[i].w - mean) * rstd * (1.f + s1.w) + s0.w;
-      const __half2 lo = __floats2half2_rn(a, b), hi = __floats2half2_rn(c, d);
-      dst[idx] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+      // warp-uniform choice of the 16-bit format (the kernel is bound by HBM, not by issue slots)
+      dst[idx] = out_bf16 ? make_uint2(pack16x2<true>(a, b), pack16x2<true>(c, d)) : make_uint2(pack16x2<false>(a, b), pack16x2<false>(c, d));
     }
   }
 }
@@ -389,7 +389,8 @@ __global__ void __launch_bounds__(kLnWarps * 32, (kLnMaxVec <= 8 ? 6 : (kLnMaxVe
 ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out, __half* __restrict__ h,
                    const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                    int T, int H, float eps, const __grid_constant__ SeqInfo seq,
-                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale, int row0) {
+                   long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale, int row0,
+                   int out_bf16) {
   // rows are local to the launch (a launch may cover a slice of the batch starting at packed row row0:
   // the data pointers are already offset, only the request lookup needs the packed index)
   const int row = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
@@ -398,7 +399,7 @@ ln_modulate_kernel(const void* __restrict__ xin, float* __restrict__ stream_out,
   const uint8_t* src = static_cast<const uint8_t*>(xin) + static_cast<size_t>(row) * H * (kFromBf16 ? 2 : 4);
   const long long voff = ln_vector_offset(seq, geo, row + row0, req_stride, kind_stride);
   ln_modulate_row<kFromBf16, kLnMaxVec, kOutFp8>(src, row, lane, stream_out, h, reinterpret_cast<const float4*>(shift0 + voff),
-                                                 reinterpret_cast<const float4*>(scale0 + voff), H, eps, row_scale);
+                                                 reinterpret_cast<const float4*>(scale0 + voff), H, eps, row_scale, out_bf16 != 0);
 }
 
 // The same rows fed by bulk copies.  Per-thread loads keep at most a few tens of KB in flight per SM
@@ -418,7 +419,7 @@ ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_
                        const float* __restrict__ shift0, const float* __restrict__ scale0, long long req_stride,
                        int T, int H, float eps, const __grid_constant__ SeqInfo seq,
                        long long kind_stride, const __grid_constant__ RowGeom geo, float* __restrict__ row_scale,
-                       int slots, int cache_vectors, int* __restrict__ status, int row0) {
+                       int slots, int cache_vectors, int* __restrict__ status, int row0, int out_bf16) {
   extern __shared__ __align__(128) uint8_t ln_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t row_bytes = static_cast<uint32_t>(H) * (kFromBf16 ? 2u : 4u);
@@ -470,7 +471,7 @@ ln_modulate_tma_kernel(const void* __restrict__ xin, float* __restrict__ stream_
           sc = reinterpret_cast<const float4*>(scale0 + voff);
         }
         ln_modulate_row<kFromBf16, kLnMaxVec, kOutFp8>(my_rows + static_cast<size_t>(slot) * row_bytes, row, lane, stream_out, h,
-                                                       sh, sc, H, eps, row_scale);
+                                                       sh, sc, H, eps, row_scale, out_bf16 != 0);
         __syncwarp();                               // every lane has read the buffer: refill it
         const int next = row + slots * kLnTmaWarps;
         if (lane == 0 && next < r1) fetch(next, slot);
@@ -532,8 +533,11 @@ pack_tokens_kernel(const __grid_constant__ PtrList src, const __grid_constant__ 
 
 // ------------------------------------------------------------------------------------------------
 // Weight load: bf16 [K, N] row-major -> fp16 [N, K] row-major (K-major B operand of the GEMMs).
-// bf16 -> fp16 is exact for |w| >= 2^-17 (8 significant bits fit fp16's normal and subnormal range).
+// bf16 -> fp16 is exact for |w| >= 2^-17 (8 significant bits fit fp16's normal and subnormal range);
+// larger magnitudes than fp16 holds clamp to its largest finite value.  kKeepBf16: the bf16 values are
+// transposed as they are (bf16-operand mode).
 // ------------------------------------------------------------------------------------------------
+template <bool kKeepBf16 = false>
 __global__ void __launch_bounds__(256)
 transpose_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __restrict__ out, int K, int N) {
   __shared__ float tile[32][33];
@@ -546,7 +550,7 @@ transpose_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __res
   __syncthreads();
   for (int i = ty; i < 32; i += 8) {
     const int n = n0 + i, k = k0 + tx;
-    if (n < N && k < K) out[static_cast<size_t>(n) * K + k] = __float2half_rn(tile[tx][i]);
+    if (n < N && k < K) reinterpret_cast<uint16_t*>(out)[static_cast<size_t>(n) * K + k] = pack16<kKeepBf16>(tile[tx][i]);
   }
 }
 
@@ -580,6 +584,28 @@ transpose_bf16_to_e4m3_kernel(const __nv_bfloat16* __restrict__ in, const float*
     if (n < N && k < K)
       out[static_cast<size_t>(n) * K + k] = static_cast<uint8_t>(__nv_cvt_float_to_fp8(tile[tx][i] / scale[n], __NV_SATFINITE, __NV_E4M3));
   }
+}
+
+// Test hooks.  fill_u32_kernel writes a 32-bit pattern (guard areas of the workspace).
+__global__ void fill_u32_kernel(uint32_t* __restrict__ dst, uint32_t value, int n) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = value;
+}
+
+// One warp waits with the library's bounded-wait routine on a barrier that nothing signals: a few
+// parked attempts, then a 50 microsecond limit on the global timer.  The wait gives up, the kernel
+// records it in the status word and returns; it holds no tensor memory and has no copy in flight.
+__global__ void __launch_bounds__(32) expire_wait_kernel(int* __restrict__ status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  const bool ok = mbar_wait_limited<2, 50000ull>(smem_u32(&bar), 0, &abort_flag);
+  __syncwarp();
+  if (threadIdx.x == 0 && (!ok || abort_flag)) atomicMax(status, kStatusTestTimeout);
 }
 
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, int n, float fill) {

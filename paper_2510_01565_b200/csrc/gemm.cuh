@@ -58,6 +58,7 @@ struct GemmParams {
   // FP8 launches only: A and Wt hold e4m3 codes; out = acc * row_scale[m] * col_scale[n] + bias
   const float* row_scale;   // [M]
   const float* col_scale;   // [N]
+  int operand_bf16;         // A and Wt hold bf16 instead of fp16 (same tensor maps: 16-bit elements)
 };
 
 namespace gemm_cfg {
@@ -107,7 +108,9 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int ban
 // geometry), everything else is unchanged.
 // FP8: both operands are e4m3 (1 byte per element, 128 elements per 128-byte swizzled row, K = 32
 // per MMA); the row and column scales that map the codes back are applied in the epilogue.
-template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false>
+// BF16: the 16-bit outputs are written as bf16 instead of fp16 (bf16-operand mode; the operands' format
+// itself is a run-time field of the instruction descriptor, p.operand_bf16).
+template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false, bool BF16 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmB2, const GemmParams p,
@@ -181,7 +184,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = FP8 ? idesc_e4m3(2 * BM, BN) : idesc_f16(2 * BM, BN, false);
+      const uint32_t idesc = FP8 ? idesc_e4m3(2 * BM, BN) : idesc_f16(2 * BM, BN, false, p.operand_bf16 != 0);
       int stage = 0; uint32_t phase = 0; int it = 0;
       for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
         const int acc = it & 1; const uint32_t acc_phase = (it >> 1) & 1u;
@@ -339,8 +342,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               uint32_t w[4];
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
-                const __half2 hh = __floats2half2_rn(v[8 * q + 2 * h], v[8 * q + 2 * h + 1]);
-                w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+                w[h] = pack16x2<BF16>(v[8 * q + 2 * h], v[8 * q + 2 * h + 1]);
               }
               dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
             }
@@ -418,8 +420,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (FP8) { ab.x *= sa * __ldg(p.col_scale + col0 + i); ab.y *= sa * __ldg(p.col_scale + col0 + i + 1); }
                 ab = fadd2(ab, bb[h]);
                 if (EPI == kEpiBiasGeluF16) ab = gelu_tanh_f32x2(ab);
-                const __half2 hh = __floats2half2_rn(ab.x, ab.y);
-                w[h] = *reinterpret_cast<const uint32_t*>(&hh);
+                w[h] = pack16x2<BF16>(ab.x, ab.y);
               }
               srow[v] = make_uint4(w[0], w[1], w[2], w[3]);
             }
@@ -443,7 +444,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (FP8) a *= sa * p.col_scale[col0 + i];
                 a += bias[col0 + i];
                 if (EPI == kEpiBiasGeluF16) a = gelu_tanh_f32(a);
-                dst[i] = __float2half_rn(a);
+                reinterpret_cast<uint16_t*>(dst)[i] = pack16<BF16>(a);
               }
             }
           }

@@ -79,24 +79,30 @@ constexpr uint64_t kWaitLimitNs = 4000000000ull;
 
 // Bounded wait.  Returns false when `*abort_flag` (shared memory, set by any thread of the CTA
 // that gave up) is raised or the limit ran out; in the latter case it raises the flag itself.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// kParkedTries: event-driven try_wait attempts before the timer is consulted; kLimitNs: wall-time
+// limit of the polling phase that follows.
+template <int kParkedTries, uint64_t kLimitNs>
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   // try_wait suspends the thread in hardware until the phase completes or a short system limit
   // passes, so this loop is not a hot spin; the timer, the abort flag and the back-off only come
   // into play for waits far longer than any healthy one.
   if (mbar_test_wait(bar, parity)) return true;          // already complete: no suspension round trip
-  for (int i = 0; i < (1 << 16); ++i)
+  for (int i = 0; i < kParkedTries; ++i)
     if (mbar_try_wait_hint(bar, parity, DIT_MBAR_SUSPEND_NS)) return true;
   const uint64_t t0 = global_ns();
   while (true) {
     for (int i = 0; i < 1024; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) {
+    if (global_ns() - t0 > kLimitNs) {
       *abort_flag = 1;
       return false;
     }
     __nanosleep(64);
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limited<(1 << 16), kWaitLimitNs>(bar, parity, abort_flag);
 }
 
 // One-dimensional bulk copy global -> shared (no tensor map): both addresses 16-byte aligned, size a
@@ -325,6 +331,24 @@ __device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
       : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
   return *reinterpret_cast<float2*>(&d);
 }
+// Two fp32 values -> one packed pair of 16-bit floats (`lo` in the low half), round to nearest even.
+// Magnitudes beyond the largest finite value of the format clamp to it instead of becoming infinite:
+// an out-of-range activation then stays a (wrong but) finite number and cannot turn into NaN in a
+// neighbouring request through 0 * inf.  BF16 selects bfloat16, else fp16.
+template <bool BF16 = false>
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi) {
+  uint32_t r;
+  if (BF16) asm("cvt.rn.satfinite.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+template <bool BF16 = false>
+__device__ __forceinline__ uint16_t pack16(float x) {
+  uint16_t r;
+  if (BF16) asm("cvt.rn.satfinite.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
+  else asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(r) : "f"(x));
+  return r;
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -345,10 +369,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   return d;
 }
 
-// Instruction descriptor for kind::f16: D fp32, A/B fp16, A K-major; B K-major or MN-major.
-__host__ __device__ constexpr uint32_t idesc_f16(int m, int n, bool b_mn_major) {
+// Instruction descriptor for kind::f16: D fp32, A/B fp16 (or both bf16), A K-major; B K-major or MN-major.
+__host__ __device__ constexpr uint32_t idesc_f16(int m, int n, bool b_mn_major, bool bf16 = false) {
   return (1u << 4)                              // D format fp32
-         | (0u << 7) | (0u << 10)               // A, B format fp16
+         | ((bf16 ? 1u : 0u) << 7) | ((bf16 ? 1u : 0u) << 10)   // A, B format: 0 = fp16, 1 = bf16
          | (0u << 15)                           // A K-major
          | ((b_mn_major ? 1u : 0u) << 16)       // B major
          | (static_cast<uint32_t>(n >> 3) << 17)

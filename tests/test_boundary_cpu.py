@@ -73,10 +73,12 @@ def test_workspace_bytes_and_config_validation(lib):
     assert ws(max_blocks=8) - full >= 4 * 18 * 3072 * 3072 * 2
     assert ws(max_total_tokens=2 * 9216) > full
     for bad in [dict(hidden=3000), dict(head_dim=96, n_heads=32), dict(n_heads=23), dict(mlp_hidden=100),
-                dict(max_requests=65), dict(max_requests=0), dict(max_blocks=0), dict(flags=8), dict(hidden=8192, n_heads=64),
+                dict(max_requests=65), dict(max_requests=0), dict(max_blocks=0), dict(flags=16), dict(hidden=8192, n_heads=64),
+                dict(flags=8 | 1), dict(flags=8 | 2), dict(flags=8 | 4),     # bf16 operands: plain blocks only
                 dict(ln_eps=-1.0)]:
         assert ws(**bad) == 0, bad
     assert ws(flags=7) == full        # the variant bits are accepted and cost no workspace
+    assert ws(flags=8) == full        # so is the bf16-operand mode (same element sizes)
     assert lib.dit_workspace_bytes(None) == 0
 
 

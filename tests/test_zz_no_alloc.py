@@ -5,11 +5,12 @@ runtime's execution phase, or a process whose GPU memory pool is owned by a fram
 out as fixed buffers.  `dit_modulation_noalloc` serves them: it takes only caller buffers and
 keeps its one piece of scratch (the fp32 bias) in a fixed array inside the library.  This test calls
 it through the C ABI twice in a row with different inputs and compares each result with the `mod`
-vectors that `dit_step_forward` computes for the same block.
+vectors that `dit_step_forward` computes for the same block, and with the CPU oracle's.
 """
 import numpy as np
 import pytest
 
+from oracle import dit_oracle as O
 from paper_2510_01565_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -56,6 +57,14 @@ def test_noalloc_modulation_matches_context_path_twice():
     assert _rel(got0, ref[:, 0]) <= TOL
     assert _rel(got1, ref[:, 1]) <= TOL
     assert np.abs(got0 - got1).max() > 1e-3        # the two calls really computed different blocks
+    # and directly against the oracle's modulation vectors (block 1 without its bias)
+    for r in range(R):
+        c = W.bf16_to_f64(wl.cond[r])
+        w0, w1 = ({k: W.bf16_to_f64(v) for k, v in wl.weights[b].items()} for b in (0, 1))
+        want0 = np.concatenate(O.adaln_modulation(c, w0["w_ada"], w0["b_ada"]))
+        want1 = np.concatenate(O.adaln_modulation(c, w1["w_ada"], np.zeros_like(w1["b_ada"])))
+        assert _rel(got0[r], want0) <= TOL
+        assert _rel(got1[r], want1) <= TOL
     ctx.close()
 
 
@@ -72,5 +81,9 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
     assert lib.dit_modulation_noalloc(p, p, None, 1, 64, 100, p, None) == 2        # unsupported hidden
     assert lib.dit_modulation_noalloc(None, p, None, 1, 64, 64, p, None) == 1
     assert lib.dit_modulation_noalloc(None, None, None, 0, 64, 64, None, None) == 0
+    # W_ada is read with 16-byte loads: a view that starts 2 bytes into a buffer is refused on the host
+    odd = C.c_void_p(buf.data_ptr() + 2)
+    assert lib.dit_modulation_noalloc(p, odd, None, 1, 64, 64, p, None) == 1
+    assert lib.dit_modulation_noalloc(p, p, None, 1, 64, 64, odd, None) == 1       # fp32 output at an odd half-word
     torch.cuda.synchronize()
     assert float(buf.abs().max()) == 0.0           # nothing was launched by the rejected calls
