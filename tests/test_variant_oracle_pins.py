@@ -300,3 +300,72 @@ def test_fp8_block_is_the_plain_block_with_two_products_swapped():
     assert np.array_equal(taps8["h1"], taps["h1"])                          # LayerNorm is untouched
     assert np.array_equal(taps8["qkv"], O.fp8_linear(taps["h1"], w["w_qkv"], w["b_qkv"]))
     assert 1e-4 < O.error_metric(y8, y) < 0.2
+
+
+# ----------------------------------------------------------------------------- e4m3 operands for all four products
+def test_fp8_all_products_block_is_the_plain_block_with_four_products_swapped():
+    from oracle import fp8_oracle as F8
+    rng = np.random.default_rng(3)
+    H, F, C, heads, L = 64, 128, 8, 2, 7
+    w = _block(rng, H, F, C)
+    w["b_o"], w["b_fc2"] = rng.standard_normal(H) * 0.1, rng.standard_normal(H) * 0.1
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    # quantising no product is the exact block; quantising QKV and the up-projection is dit_oracle's fp8=True
+    assert np.array_equal(F8.block_forward_fp8(x, cond, w, heads, 1e-6, quantise=()), O.block_forward(x, cond, w, heads, 1e-6))
+    assert np.array_equal(F8.block_forward_fp8(x, cond, w, heads, 1e-6, quantise=("qkv", "fc1")),
+                          O.block_forward(x, cond, w, heads, 1e-6, fp8=True))
+    # each product of the all-four block is fp8_linear of the tap that feeds it
+    t = {}
+    y = F8.block_forward_fp8(x, cond, w, heads, 1e-6, taps=t)
+    m = O.adaln_modulation(cond, w["w_ada"], w["b_ada"])
+    assert np.array_equal(t["qkv"], O.fp8_linear(t["h1"], w["w_qkv"], w["b_qkv"]))
+    assert np.array_equal(t["x_mid"], x + m[2] * O.fp8_linear(t["a"], w["w_o"], w["b_o"]))
+    assert np.array_equal(t["u"], O.gelu_tanh(O.fp8_linear(t["h2"], w["w_fc1"], w["b_fc1"])))
+    assert np.array_equal(y, t["x_mid"] + m[5] * O.fp8_linear(t["u"], w["w_fc2"], w["b_fc2"]))
+    # a few per cent from the exact block, and further from it than the two-product form
+    exact = O.block_forward(x, cond, w, heads, 1e-6)
+    e4, e2 = O.error_metric(y, exact), O.error_metric(O.block_forward(x, cond, w, heads, 1e-6, fp8=True), exact)
+    assert 1e-3 < e4 < 0.3 and e2 < 0.3
+    # row subset, stack and packed step are consistent with one another
+    rows = np.array([0, 3, 6])
+    assert np.allclose(F8.block_forward_fp8(x, cond, w, heads, 1e-6, rows=rows), y[rows], rtol=1e-12, atol=1e-12)
+    w2 = _block(rng, H, F, C)
+    two = F8.stack_forward_fp8(x, cond, [w, w2], heads, 1e-6)
+    assert np.array_equal(two, F8.block_forward_fp8(y, cond, w2, heads, 1e-6))
+    packed = np.concatenate([x, x[:3]])
+    step = F8.step_forward_fp8(packed, [L, 3], np.stack([cond, cond * 0.5]), [w, w2], heads, 1e-6)
+    assert np.array_equal(step[:L], two)
+    assert np.array_equal(step[L:], F8.stack_forward_fp8(x[:3], cond * 0.5, [w, w2], heads, 1e-6))
+
+
+def test_fp8_all_products_is_exact_when_every_operand_sits_on_the_grid():
+    """Weights on the e4m3 grid with a column maximum of 448 * 2^k lose nothing; an output projection
+    whose left operand rows are on the grid too is then exact, which pins that the scales are removed
+    again (a missing or doubled scale would be off by the scale itself)."""
+    from oracle import fp8_oracle as F8
+    rng = np.random.default_rng(4)
+    a = O.quantize_e4m3(rng.uniform(-448, 448, (6, 32))) * 2.0 ** -9
+    a[:, 0] = 448.0 * 2.0 ** -9                           # every row's maximum maps to 448 exactly
+    w_o = O.quantize_e4m3(rng.uniform(-448, 448, (32, 32))) * 2.0 ** -12
+    w_o[0, :] = -448.0 * 2.0 ** -12
+    assert np.allclose(O.fp8_linear(a, w_o, np.zeros(32)), a @ w_o, rtol=1e-14, atol=0)
+
+
+def test_fp8_parallel_block_concatenates_before_it_scales():
+    from oracle import fp8_oracle as F8
+    rng = np.random.default_rng(5)
+    H, F, C, heads, L = 64, 128, 8, 2, 5
+    w = {"w_ada": rng.standard_normal((C, 3 * H)) * 0.1, "b_ada": rng.standard_normal(3 * H) * 0.1,
+         "w_qkv": rng.standard_normal((H, 3 * H)) * 0.2, "b_qkv": rng.standard_normal(3 * H) * 0.1,
+         "w_fc1": rng.standard_normal((H, F)) * 0.2, "b_fc1": rng.standard_normal(F) * 0.1,
+         "w_out": rng.standard_normal((H + F, H)) * 0.2, "b_out": rng.standard_normal(H) * 0.1}
+    x, cond = rng.standard_normal((L, H)), rng.standard_normal(C)
+    t = {}
+    y = F8.parallel_block_forward_fp8(x, cond, w, heads, 1e-6, taps=t)
+    gate = np.split(O.silu(cond) @ w["w_ada"] + w["b_ada"], 3)[2]
+    cat = np.concatenate([t["a"], t["u"]], axis=1)
+    assert np.array_equal(y, x + gate * O.fp8_linear(cat, w["w_out"], w["b_out"]))
+    # one scale per concatenated row: scaling the attention half by 2^6 changes how the MLP half is rounded
+    exact = O.parallel_block_forward(x, cond, w, heads, 1e-6)
+    assert 1e-3 < O.error_metric(y, exact) < 0.3
+    assert np.array_equal(F8.stack_forward_fp8(x, cond, [w], heads, 1e-6), y)
