@@ -233,7 +233,9 @@ class DeviceBench:
         flops = {"gemm_qkv": 2.0 * T * H * 3 * H, "gemm_proj": 2.0 * T * H * H, "gemm_fc1": 2.0 * T * H * F,
                  "gemm_fc2": 2.0 * T * H * (F + (H if self.form == "parallel" else 0)),   # parallel form: one K = H + F output GEMM
                  "attention": 4.0 * H * sum(l * l for l in self.lens)}
-        nbytes = {"ln_modulate": T * H * (4 + 2), "modulation": self.slots * wl.dims.cond_dim * 6 * H * 2}
+        nbytes = {"ln_modulate": T * H * (4 + 2), "modulation": self.slots * wl.dims.cond_dim * 6 * H * 2,
+                  # e4m3 mode: fp16 in, codes out, two launches per block (attention output, GELU output; one for a parallel block)
+                  "quantize": T * (H + F) * 3 / (1 if self.form == "parallel" else 2)}
         kern = {}
         for name, rec in kernels.items():
             if not rec["launches"]:
@@ -503,7 +505,7 @@ def run_gpu(args):
             "dtype": dtype, "data": "synthetic",
             "config": {"workload": wl.name, "block_form": args.form,
                        "block_variants": {"qk_rmsnorm": bool(args.variants & 1), "rope_2d": bool(args.variants & 2),
-                                          "fp8_qkv_fc1": bool(args.variants & 4), "bf16_operands": bool(args.variants & 8)},
+                                          "fp8_all_gemms": bool(args.variants & 4), "bf16_operands": bool(args.variants & 8)},
                        "n_blocks": nb, "weights_reused_cyclically": bool(args.depth),
                        "requests": [f"{r.height}x{r.width}+{r.n_text_tokens}" for r in wl.requests],
                        "total_tokens": T, "image_tokens": wl.image_tokens, "hidden": H, "heads": wl.dims.n_heads,

@@ -85,12 +85,13 @@ typedef struct {
  *                        or dit_denoise_step (dit_step_forward returns DIT_ERR_INVALID_ARG). */
 #define DIT_FLAG_QK_RMSNORM 1u
 #define DIT_FLAG_ROPE_2D 2u
-/* Reduced-precision mode, off in every benchmark configuration: the two GEMMs that read a LayerNorm
- * output (QKV projection and MLP up-projection, 7/12 of a block's linear FLOPs) take e4m3 operands.
- * Each row of the modulated LayerNorm output is scaled so that its largest magnitude maps to 448 and
- * rounded to e4m3 by the LayerNorm kernel; each output channel of W_qkv / W_fc1 likewise at load time;
- * the accumulator (fp32, exact products) is scaled back in the epilogue.  Everything else stays as
- * it is.  Errors grow to a few per cent of the output's rms; not available for two-stream blocks. */
+/* Reduced-precision mode, off in every benchmark configuration: the four GEMMs of a block take e4m3
+ * operands.  Each row of a left operand is scaled so that its largest magnitude maps to 448 and rounded
+ * to e4m3: the modulated LayerNorm outputs by the LayerNorm kernel itself, the attention output and the
+ * GELU output (which are produced tile by tile) by a row-quantisation pass of their own; each output
+ * channel of the four weight matrices likewise at load time; the accumulator (fp32, exact products) is
+ * scaled back in the epilogue.  Everything else stays as it is.  Errors grow to several per cent of the
+ * output's rms; not available for two-stream blocks. */
 #define DIT_FLAG_FP8_GEMM 4u
 /* bf16 operands instead of fp16: the weights are kept as given (no conversion), the 16-bit
  * activations (LayerNorm outputs, q/k/v, attention probabilities and output, GELU output) are stored
@@ -248,7 +249,9 @@ dit_status dit_debug_expire_wait(dit_ctx *ctx, void *stream);
  * entries) and starts a new accumulation. */
 typedef enum {
   DIT_KERNEL_MODULATION = 0, DIT_KERNEL_LN_MODULATE = 1, DIT_KERNEL_GEMM_QKV = 2, DIT_KERNEL_ATTENTION = 3,
-  DIT_KERNEL_GEMM_PROJ = 4, DIT_KERNEL_GEMM_FC1 = 5, DIT_KERNEL_GEMM_FC2 = 6, DIT_KERNEL_KINDS = 7
+  DIT_KERNEL_GEMM_PROJ = 4, DIT_KERNEL_GEMM_FC1 = 5, DIT_KERNEL_GEMM_FC2 = 6,
+  DIT_KERNEL_QUANTIZE = 7, /* e4m3 mode only: row quantisation of the attention and GELU outputs */
+  DIT_KERNEL_KINDS = 8
 } dit_kernel_kind;
 dit_status dit_ctx_set_timing(dit_ctx *ctx, int32_t enabled);
 dit_status dit_ctx_read_timing(dit_ctx *ctx, double *ms_by_kernel, int64_t *launches_by_kernel);

@@ -22,7 +22,7 @@ DIT_FLAG_FP8_GEMM = 4
 DIT_FLAG_BF16_OPERANDS = 8
 STATUS_NAMES = ["DIT_OK", "DIT_ERR_INVALID_ARG", "DIT_ERR_SHAPE", "DIT_ERR_CAPACITY", "DIT_ERR_NOT_LOADED",
                 "DIT_ERR_UNSUPPORTED_ARCH", "DIT_ERR_CUDA", "DIT_ERR_TIMEOUT", "DIT_ERR_INTERNAL"]
-KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2"]
+KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "quantize"]
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights", "dit_load_dual_block_weights",

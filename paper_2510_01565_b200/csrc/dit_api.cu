@@ -29,7 +29,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets (bytes) inside one block's weight slot.
 struct BlockLayout {
   size_t w_ada, b_ada, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, q_norm, k_norm;
-  size_t s_qkv, s_fc1;   // per-output-channel scales of the e4m3 weights (DIT_FLAG_FP8_GEMM)
+  size_t s_qkv, s_fc1, s_o, s_fc2;   // per-output-channel scales of the e4m3 weights (DIT_FLAG_FP8_GEMM)
   size_t bytes;
 };
 // Offsets (bytes) inside the workspace.
@@ -41,6 +41,8 @@ struct Layout {
   size_t sh_temb, sh_pre1, sh_cond, sh_modfin, sh_vtok, sh_pooled;
   size_t rope_theta;   // pair frequencies of one rotary axis group, fp32
   size_t row_scale;    // per-row scales of the e4m3 activations (DIT_FLAG_FP8_GEMM)
+  size_t q8, row_scale2;   // e4m3 codes [T, H + F] and row scales of the operands quantised by a pass of their own
+                           // (attention output, GELU output, or both side by side); empty without DIT_FLAG_FP8_GEMM
   size_t items;        // two-stream launches: [0] item count, then per-tile flags, then the items
   // test hooks: 1 KiB guard areas after the activation regions, and the [begin, end) ranges that
   // dit_debug_poison fills
@@ -91,6 +93,8 @@ Layout make_layout(const dit_config& c) {
   L.blk.k_norm = take(c.head_dim * 4);
   L.blk.s_qkv = take(3 * H * 4);
   L.blk.s_fc1 = take(F * 4);
+  L.blk.s_o = take(H * 4);
+  L.blk.s_fc2 = take(H * 4);
   L.blk.bytes = o;
   o = 0;
   // every activation region (or run of regions) is followed by a guard area and is listed as a poison range
@@ -136,6 +140,9 @@ Layout make_layout(const dit_config& c) {
   guard(L.sh_temb);
   L.rope_theta = take(64 * 4);
   L.row_scale = take(T * 4);
+  const bool fp8_mode = (c.flags & DIT_FLAG_FP8_GEMM) != 0;
+  L.row_scale2 = take(fp8_mode ? T * 4 : 0);
+  L.q8 = take(fp8_mode ? T * (H + F) : 0);
   guard(L.row_scale);
   L.items = take((16 + 3 * (T / (2 * 128) + 2)) * 4);
   L.bytes = o;
@@ -375,6 +382,18 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   float* row_scale = ctx->at<float>(ctx->lay.row_scale);
   if (fp8 && !make_map8(ctx, &tm_h, h, H, T, gemm_cfg::BM))   // h holds e4m3 codes in this mode
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  // e4m3 mode: the operands that are produced tile by tile (attention output, GELU output, or the two side by
+  // side in a parallel block) are quantised row by row into q8 by a pass of their own before the GEMM that reads them
+  uint8_t* q8 = ctx->at<uint8_t>(ctx->lay.q8);
+  float* row_scale2 = ctx->at<float>(ctx->lay.row_scale2);
+  CUtensorMap tm_a8, tm_u8, tm_cat8;
+  if (fp8 && (!make_map8(ctx, &tm_a8, q8, H, T, gemm_cfg::BM) || !make_map8(ctx, &tm_u8, q8, F, T, gemm_cfg::BM) ||
+              !make_map8(ctx, &tm_cat8, q8, H + F, T, gemm_cfg::BM)))
+    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  auto quantise_rows = [&](const __half* src, long long ld, int K) -> cudaError_t {
+    quantize_rows_e4m3_kernel<<<(T + kQuantWarps - 1) / kQuantWarps, kQuantWarps * 32, 0, st>>>(src, ld, q8, row_scale2, T, K);
+    return cudaGetLastError();
+  };
 
   int64_t launches = 0;
   const long long req_stride = static_cast<long long>(n_blocks) * 6 * H;
@@ -402,9 +421,14 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
 
   // The gated-residual GEMM that writes `out`, sliced by rows when the result goes to the host.  A slice is a
   // whole number of 256-row tiles; every output element is computed exactly as in the unsliced launch.
+  // In the e4m3 mode A is the quantised copy q8 (1 byte per element) and g carries the row and column scales.
   auto last_gemm = [&](const __half* a_ptr, int K, const CUtensorMap& tmA_full, const CUtensorMap& tmB, const GemmParams& g) -> dit_status {
+    auto launch = [&](const CUtensorMap& tmA, const GemmParams& q) {
+      return fp8 ? launch_gemm<kEpiGateResidF32, 0, false, true>(ctx, tmA, tmB, q, seq, st)
+                 : launch_gemm<kEpiGateResidF32>(ctx, tmA, tmB, q, seq, st);
+    };
     if (!host_out) {
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tmA_full, tmB, g, seq, st); }));
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch(tmA_full, g); }));
       return DIT_OK;
     }
     const int tile_rows = 2 * gemm_cfg::BM;
@@ -412,13 +436,15 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
       const int rows = std::min(per, T - r0);
       CUtensorMap tmA;
-      if (!make_map(ctx, &tmA, a_ptr + static_cast<size_t>(r0) * K, K, rows, gemm_cfg::BM))
+      if (!(fp8 ? make_map8(ctx, &tmA, q8 + static_cast<size_t>(r0) * K, K, rows, gemm_cfg::BM)
+                : make_map(ctx, &tmA, a_ptr + static_cast<size_t>(r0) * K, K, rows, gemm_cfg::BM)))
         return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
       GemmParams q = g;
       q.M = rows; q.row0 = r0;
       q.resid = g.resid + static_cast<size_t>(r0) * g.N;
       q.out32 = g.out32 + static_cast<size_t>(r0) * g.N;
-      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tmA, tmB, q, seq, st); }));
+      if (fp8) q.row_scale = g.row_scale + r0;
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch(tmA, q); }));
       DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->slice_done[sidx], st));
       DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->slice_done[sidx], 0));
       DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out + static_cast<size_t>(r0) * g.N, g.out32 + static_cast<size_t>(r0) * g.N,
@@ -578,11 +604,18 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       g.bias = reinterpret_cast<const float*>(wb + ctx->lay.blk.b_fc2);
       g.resid = stream; g.out32 = last ? out : stream;
       g.gate = modb + 2 * H; g.gate_stride = req_stride;
+      if (fp8) {
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_QUANTIZE, [&] { return quantise_rows(cat, H + F, H + F); }));
+        g.row_scale = row_scale2; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc2);
+      }
       if (last) {
-        const dit_status ls = last_gemm(cat, H + F, tm_cat, bs.tm_fc2, g);
+        const dit_status ls = last_gemm(cat, H + F, fp8 ? tm_cat8 : tm_cat, bs.tm_fc2, g);
         if (ls != DIT_OK) return ls;
       } else {
-        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st); }));
+        DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] {
+          return fp8 ? launch_gemm<kEpiGateResidF32, 0, false, true>(ctx, tm_cat8, bs.tm_fc2, g, seq, st)
+                     : launch_gemm<kEpiGateResidF32>(ctx, tm_cat, bs.tm_fc2, g, seq, st);
+        }));
       }
       continue;
     }
@@ -643,7 +676,12 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.resid = stream; g.out32 = stream;
     g.gate = modb + 2 * H; g.gate_stride = req_stride;
     two_stream(g, ctx->lay.blk.b_o);
+    if (fp8) {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_QUANTIZE, [&] { return quantise_rows(a, H, H); }));
+      g.row_scale = row_scale2; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_o);
+    }
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_PROJ, [&] {
+      if (fp8) return launch_gemm<kEpiGateResidF32, 0, false, true>(ctx, tm_a8, bs.tm_o, g, seq, st);
       return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_a, bs.tm_o, g, seq, st, rg, &bt.tm_o)
                   : launch_gemm<kEpiGateResidF32>(ctx, tm_a, bs.tm_o, g, seq, st);
     }));
@@ -674,9 +712,15 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     g.resid = stream; g.out32 = last ? out : stream;
     g.gate = modb + 5 * H; g.gate_stride = req_stride;
     two_stream(g, ctx->lay.blk.b_fc2);
+    if (fp8) {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_QUANTIZE, [&] { return quantise_rows(u, F, F); }));
+      g.row_scale = row_scale2; g.col_scale = reinterpret_cast<const float*>(wb + ctx->lay.blk.s_fc2);
+    }
     if (last && !dual) {
-      const dit_status ls = last_gemm(u, F, tm_u, bs.tm_fc2, g);
+      const dit_status ls = last_gemm(u, F, fp8 ? tm_u8 : tm_u, bs.tm_fc2, g);
       if (ls != DIT_OK) return ls;
+    } else if (fp8) {
+      DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] { return launch_gemm<kEpiGateResidF32, 0, false, true>(ctx, tm_u8, bs.tm_fc2, g, seq, st); }));
     } else {
       DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_GEMM_FC2, [&] {
         return dual ? launch_gemm<kEpiGateResidF32, 0, true>(ctx, tm_u, bs.tm_fc2, g, seq, st, rg, &bt.tm_fc2)
@@ -783,6 +827,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32, 0, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 128, true>), gemm_cfg::SMEM_BYTES);
+  opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiGateResidF32, 0, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasF16, 0, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiBiasGeluF16, 0, false, true>), gemm_cfg::SMEM_BYTES);
   opt_in(reinterpret_cast<const void*>(&gemm_tcgen05_kernel<kEpiQkvF16, 64, false, true>), gemm_cfg::SMEM_BYTES);
@@ -902,19 +947,19 @@ dit_status dit_load_block_weights(dit_ctx* ctx, int32_t b, const dit_block_weigh
   DIT_CUDA_TRY(ctx, bias(w->b_ada, L.b_ada, 6 * H));
   DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_qkv, L.w_qkv, L.s_qkv, H, 3 * H) : weight(w->w_qkv, L.w_qkv, H, 3 * H));
   DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
-  DIT_CUDA_TRY(ctx, weight(w->w_o, L.w_o, H, H));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_o, L.w_o, L.s_o, H, H) : weight(w->w_o, L.w_o, H, H));
   DIT_CUDA_TRY(ctx, bias(w->b_o, L.b_o, H));
   DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_fc1, L.w_fc1, L.s_fc1, H, F) : weight(w->w_fc1, L.w_fc1, H, F));
   DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
-  DIT_CUDA_TRY(ctx, weight(w->w_fc2, L.w_fc2, F, H));
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_fc2, L.w_fc2, L.s_fc2, F, H) : weight(w->w_fc2, L.w_fc2, F, H));
   DIT_CUDA_TRY(ctx, bias(w->b_fc2, L.b_fc2, H));
   DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));   // NULL scale = ones
   DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
 
   if (!(fp8 ? make_map8(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2)) ||
-      !make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) ||
+      !(fp8 ? make_map8(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_o, base + L.w_o, H, H, gemm_cfg::BN / 2)) ||
       !(fp8 ? make_map8(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2)) ||
-      !make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2))
+      !(fp8 ? make_map8(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc2, base + L.w_fc2, F, H, gemm_cfg::BN / 2)))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;
   return DIT_OK;
@@ -981,13 +1026,13 @@ dit_status dit_load_parallel_block_weights(dit_ctx* ctx, int32_t b, const dit_pa
   DIT_CUDA_TRY(ctx, bias(w->b_qkv, L.b_qkv, 3 * H));
   DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_fc1, L.w_fc1, L.s_fc1, H, F) : weight(w->w_fc1, L.w_fc1, H, F));
   DIT_CUDA_TRY(ctx, bias(w->b_fc1, L.b_fc1, F));
-  DIT_CUDA_TRY(ctx, weight(w->w_out, L.w_o, H + F, H));          // runs on over the W_fc2 region
+  DIT_CUDA_TRY(ctx, fp8 ? weight8(w->w_out, L.w_o, L.s_fc2, H + F, H) : weight(w->w_out, L.w_o, H + F, H));   // runs on over the W_fc2 region
   DIT_CUDA_TRY(ctx, bias(w->b_out, L.b_fc2, H));
   DIT_CUDA_TRY(ctx, bias(w->q_norm, L.q_norm, ctx->cfg.head_dim, 1.f));
   DIT_CUDA_TRY(ctx, bias(w->k_norm, L.k_norm, ctx->cfg.head_dim, 1.f));
   if (!(fp8 ? make_map8(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_qkv, base + L.w_qkv, H, 3 * H, gemm_cfg::BN / 2)) ||
       !(fp8 ? make_map8(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc1, base + L.w_fc1, H, F, gemm_cfg::BN / 2)) ||
-      !make_map(ctx, &bs.tm_fc2, base + L.w_o, H + F, H, gemm_cfg::BN / 2))
+      !(fp8 ? make_map8(ctx, &bs.tm_fc2, base + L.w_o, H + F, H, gemm_cfg::BN / 2) : make_map(ctx, &bs.tm_fc2, base + L.w_o, H + F, H, gemm_cfg::BN / 2)))
     return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
   bs.loaded = true;
   return DIT_OK;

@@ -568,6 +568,47 @@ col_absmax_scale_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict_
   scale[n] = amax > 0.f ? amax / 448.0f : 1.0f;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Row quantisation for the e4m3 mode: fp16 rows [T, K] (row stride ld elements) -> e4m3 codes [T, K]
+// (dense) and one scale per row, largest magnitude of the row -> 448.  Used for the operands that are
+// produced tile by tile (attention output, GELU output), where no kernel sees a whole row: one warp
+// per row, two sweeps (the second one finds the row in L1/L2).  Bound by HBM: 3 bytes per element.
+// ------------------------------------------------------------------------------------------------
+constexpr int kQuantWarps = 8;
+
+__global__ void __launch_bounds__(kQuantWarps * 32)
+quantize_rows_e4m3_kernel(const __half* __restrict__ in, long long ld, uint8_t* __restrict__ out,
+                          float* __restrict__ row_scale, int T, int K) {
+  const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= T) return;
+  const uint4* src = reinterpret_cast<const uint4*>(in + static_cast<size_t>(row) * ld);   // 8 values per load
+  const int nvec = K >> 3;
+  __half2 m2 = __float2half2_rn(0.f);
+  for (int i = lane; i < nvec; i += 32) {
+    const uint4 v = src[i];
+    const __half2* h2 = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) m2 = __hmax2(m2, __habs2(h2[q]));
+  }
+  float amax = fmaxf(__low2float(m2), __high2float(m2));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
+  if (lane == 0) row_scale[row] = amax > 0.f ? amax / 448.0f : 1.0f;
+  uint2* dst = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * K);
+  for (int i = lane; i < nvec; i += 32) {
+    const uint4 v = src[i];
+    const __half2* h2 = reinterpret_cast<const __half2*>(&v);
+    uint32_t c[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 f = __half22float2(h2[q]);
+      c[q] = __nv_cvt_float2_to_fp8x2(make_float2(f.x * inv, f.y * inv), __NV_SATFINITE, __NV_E4M3);
+    }
+    dst[i] = make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+  }
+}
+
 __global__ void __launch_bounds__(256)
 transpose_bf16_to_e4m3_kernel(const __nv_bfloat16* __restrict__ in, const float* __restrict__ scale,
                               uint8_t* __restrict__ out, int K, int N) {

@@ -234,12 +234,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const bool one_req = __all_sync(0xffffffffu, my_req == req0 || my_req < 0);
       // fp32 epilogues: this lane stores columns (lane % 8) * 4 .. + 3 of rows it * 4 + lane / 8, it < 8
       int row_req[8];
+      float row_sa[8];                       // FP8: the row scales of the rows this lane stores
       unsigned store_rows = 0;
       if (EPI == kEpiGateResidF32 || EPI == kEpiBiasF32) {
 #pragma unroll
         for (int i8 = 0; i8 < 8; ++i8) {
           const int rr = i8 * 4 + (lane >> 3);
           row_req[i8] = __shfl_sync(0xffffffffu, my_req, rr);
+          if (FP8) row_sa[i8] = __shfl_sync(0xffffffffu, sa, rr);
           const int rk = DUAL ? __shfl_sync(0xffffffffu, my_kind, rr) : 0;
           if (m0 + quarter * 32 + rr < p.M && (!DUAL || rk == kind)) store_rows |= 1u << i8;
         }
@@ -369,6 +371,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const int col = col0 + cg;                        // N is a multiple of 64: the whole chunk is inside
           {
             const float4 b = __ldg(reinterpret_cast<const float4*>(bias + col));
+            float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
+            if (FP8) cs = __ldg(reinterpret_cast<const float4*>(p.col_scale + col));
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
             if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(gate + req0 * p.gate_stride + col));
             float4 x[8];
@@ -384,8 +388,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               if ((store_rows >> it) & 1u) {
                 if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(gate + row_req[it] * p.gate_stride + col));
                 const float4 a = *reinterpret_cast<const float4*>(st + rr * 36 + cg);
-                const float2 s0 = fadd2(make_float2(a.x, a.y), make_float2(b.x, b.y));
-                const float2 s1 = fadd2(make_float2(a.z, a.w), make_float2(b.z, b.w));
+                float2 s0, s1;
+                if (FP8) {     // codes back to values: row scale of the activations, column scale of the weights
+                  const float sr = row_sa[it];
+                  s0 = ffma2(make_float2(a.x, a.y), make_float2(sr * cs.x, sr * cs.y), make_float2(b.x, b.y));
+                  s1 = ffma2(make_float2(a.z, a.w), make_float2(sr * cs.z, sr * cs.w), make_float2(b.z, b.w));
+                } else {
+                  s0 = fadd2(make_float2(a.x, a.y), make_float2(b.x, b.y));
+                  s1 = fadd2(make_float2(a.z, a.w), make_float2(b.z, b.w));
+                }
                 float4 o;
                 if (EPI == kEpiGateResidF32) {
                   const float2 o0 = ffma2(make_float2(g.x, g.y), s0, make_float2(x[it].x, x[it].y));
