@@ -319,8 +319,8 @@ size_t mod_smem_bytes(int C) {   // activations [G][C], later reused for the sli
   return std::max<size_t>(static_cast<size_t>(kModReqGroup) * C, static_cast<size_t>(8) * kModThreads * kModReqGroup) * sizeof(float);
 }
 
-size_t mod_tma_smem_bytes(int C) {
-  return mod_tma_act_floats(C) * sizeof(float) + kModTmaRingBytes + 2 * kModTmaSlices * kModTmaStages * 8 + 16;
+size_t mod_tma_smem_bytes(int C, int G) {
+  return mod_tma_act_floats(C, G) * sizeof(float) + kModTmaRingBytes + 2 * kModTmaSlices * kModTmaStages * 8 + 16;
 }
 constexpr size_t kModTmaSmemMax = 224 * 1024;
 
@@ -331,8 +331,13 @@ constexpr size_t kModTmaSmemMax = 224 * 1024;
 cudaError_t launch_modulation(const ModParams& mp, int num_sms, size_t smem, cudaStream_t st, int* status, const CUtensorMap* tmW) {
   auto ctas = [&](int cols) { return mp.NB * ((mp.N6 + cols - 1) / cols); };
   const int enough = 3 * num_sms / 2;
-  if (status && tmW && ctas(kModTmaCols) >= enough && mod_tma_smem_bytes(mp.C) <= kModTmaSmemMax) {
-    modulation_tma_kernel<<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C), st>>>(*tmW, mp, status);
+  // the bulk-copy kernel keeps 120 KB in flight per CTA and holds an SM alone: about one CTA per SM is already enough
+  if (status && tmW && ctas(kModTmaCols) >= num_sms * 9 / 10 && mod_tma_smem_bytes(mp.C, 8) <= kModTmaSmemMax) {
+    // requests per pass over W_ada: the smallest group that covers the batch
+    if (mp.R <= 1) modulation_tma_kernel<1><<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C, 1), st>>>(*tmW, mp, status);
+    else if (mp.R <= 2) modulation_tma_kernel<2><<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C, 2), st>>>(*tmW, mp, status);
+    else if (mp.R <= 4) modulation_tma_kernel<4><<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C, 4), st>>>(*tmW, mp, status);
+    else modulation_tma_kernel<8><<<ctas(kModTmaCols), kModTmaThreads, mod_tma_smem_bytes(mp.C, 8), st>>>(*tmW, mp, status);
     return cudaGetLastError();
   }
   if (ctas(1024) >= enough) modulation_kernel<kModInCondSilu, 1024><<<ctas(1024), kModThreads, smem, st>>>(mp);
@@ -842,7 +847,10 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 256>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 512>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInCondSilu, 1024>), mod_smem_bytes(kMaxCondDim));
-  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel), kModTmaSmemMax);
+  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel<1>), kModTmaSmemMax);
+  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel<2>), kModTmaSmemMax);
+  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel<4>), kModTmaSmemMax);
+  opt_in(reinterpret_cast<const void*>(&modulation_tma_kernel<8>), kModTmaSmemMax);
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32Silu>), mod_smem_bytes(kMaxCondDim));
   opt_in(reinterpret_cast<const void*>(&modulation_kernel<kModInF32>), mod_smem_bytes(kMaxCondDim));
   {

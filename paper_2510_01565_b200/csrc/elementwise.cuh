@@ -149,18 +149,22 @@ constexpr int kModTmaCols = 512, kModTmaSlices = 4, kModTmaStages = 2, kModTmaRo
 constexpr int kModTmaComputeThreads = 256, kModTmaThreads = kModTmaComputeThreads + 32;
 constexpr int kModTmaRingBytes = kModTmaSlices * kModTmaStages * kModTmaRows * kModTmaCols * 2;
 
-__host__ __device__ inline size_t mod_tma_act_floats(int C) {      // activations [C][G], later the slice partials
-  const size_t a = static_cast<size_t>(kModReqGroup) * C, b = static_cast<size_t>(kModTmaSlices) * kModReqGroup * kModTmaCols;
-  return a > b ? a : b;
+__host__ __device__ inline size_t mod_tma_act_floats(int C, int G) {      // activations [C][G], later the slice partials
+  const size_t a = static_cast<size_t>(G) * C, b = static_cast<size_t>(kModTmaSlices) * G * kModTmaCols;
+  return ((a > b ? a : b) + 31) & ~static_cast<size_t>(31);      // the ring that follows must start on a 128-byte boundary
 }
 
+// G = requests handled per pass over W_ada (1, 2, 4 or 8; the host takes the smallest that covers the batch, so
+// that a small batch does not pay the multiply-adds of eight).  Every request has its own accumulators, so
+// its result does not depend on G or on the other requests.
+template <int G>
 __global__ void __launch_bounds__(kModTmaThreads, 1)
 modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p, int* __restrict__ status) {
-  static_assert(kModReqGroup == 8, "the activation layout below packs 8 requests per row");
+  static_assert(G == 1 || G == 2 || G == 4 || G == 8, "the activation layout packs G requests per row");
   extern __shared__ __align__(128) uint8_t mod_smem[];
-  float* s_act = reinterpret_cast<float*>(mod_smem);               // [C][8]
+  float* s_act = reinterpret_cast<float*>(mod_smem);               // [C][G]
   float* s_part = s_act;
-  uint8_t* ring = mod_smem + mod_tma_act_floats(p.C) * sizeof(float);
+  uint8_t* ring = mod_smem + mod_tma_act_floats(p.C, G) * sizeof(float);
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring + kModTmaRingBytes);      // full[slice][stage], then empty[slice][stage]
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kModTmaSlices * kModTmaStages);
   const int cols_per_block = (p.N6 + kModTmaCols - 1) / kModTmaCols;
@@ -189,11 +193,11 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
   }
   int used = 0;                                // stage uses so far (keeps the barrier phases across request groups)
   bool ok = true;
-  for (int r0 = 0; r0 < p.R; r0 += kModReqGroup) {
-    const int g = min(kModReqGroup, p.R - r0);
+  for (int r0 = 0; r0 < p.R; r0 += G) {
+    const int g = min(G, p.R - r0);
     __syncthreads();                           // barriers exist; previous group's partials have been read
-    for (int i = threadIdx.x; i < kModReqGroup * p.C; i += kModTmaThreads) {
-      const int cc = i >> 3, rr = i & 7;
+    for (int i = threadIdx.x; i < G * p.C; i += kModTmaThreads) {
+      const int cc = i / G, rr = i % G;
       float v = 0.f;
       if (rr < g) {
         const float x = __bfloat162float(p.cond[static_cast<size_t>(r0 + rr) * p.C + cc]);
@@ -220,9 +224,9 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
       used += n_groups;
     } else {
       // ------------------------------------------------------------------ compute warps
-      float2 acc[kModReqGroup][4];
+      float2 acc[G][4];
 #pragma unroll
-      for (int rr = 0; rr < kModReqGroup; ++rr)
+      for (int rr = 0; rr < G; ++rr)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[rr][q] = make_float2(0.f, 0.f);
       for (int k = 0; k < n_groups; ++k, ++used) {
@@ -239,11 +243,22 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
               float2 wf[4];
 #pragma unroll
               for (int q = 0; q < 4; ++q) wf[q] = make_float2(__uint_as_float(u4[q] << 16), __uint_as_float(u4[q] & 0xFFFF0000u));
-              const float4 a_lo = *reinterpret_cast<const float4*>(s_act + static_cast<size_t>(r_first + j) * 8);
-              const float4 a_hi = *reinterpret_cast<const float4*>(s_act + static_cast<size_t>(r_first + j) * 8 + 4);
-              const float a[8] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w, a_hi.x, a_hi.y, a_hi.z, a_hi.w};
+              float a[G];
+              const float* ap = s_act + static_cast<size_t>(r_first + j) * G;
+              if constexpr (G == 8) {
+                const float4 a_lo = *reinterpret_cast<const float4*>(ap), a_hi = *reinterpret_cast<const float4*>(ap + 4);
+                a[0] = a_lo.x; a[1] = a_lo.y; a[2] = a_lo.z; a[3] = a_lo.w; a[4] = a_hi.x; a[5] = a_hi.y; a[6] = a_hi.z; a[7] = a_hi.w;
+              } else if constexpr (G == 4) {
+                const float4 a4 = *reinterpret_cast<const float4*>(ap);
+                a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
+              } else if constexpr (G == 2) {
+                const float2 a2 = *reinterpret_cast<const float2*>(ap);
+                a[0] = a2.x; a[1] = a2.y;
+              } else {
+                a[0] = *ap;
+              }
 #pragma unroll
-              for (int rr = 0; rr < kModReqGroup; ++rr) {
+              for (int rr = 0; rr < G; ++rr) {
                 const float2 aa = make_float2(a[rr], a[rr]);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) acc[rr][q] = ffma2(aa, wf[q], acc[rr][q]);
@@ -258,11 +273,11 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
       // the partials go into the activation buffer once every compute warp has finished with it (below)
       asm volatile("bar.sync 1, %0;" ::"n"(kModTmaComputeThreads));
 #pragma unroll
-      for (int rr = 0; rr < kModReqGroup; ++rr)
+      for (int rr = 0; rr < G; ++rr)
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          s_part[(slice * kModReqGroup + rr) * kModTmaCols + cg * 8 + 2 * q] = acc[rr][q].x;
-          s_part[(slice * kModReqGroup + rr) * kModTmaCols + cg * 8 + 2 * q + 1] = acc[rr][q].y;
+          s_part[(slice * G + rr) * kModTmaCols + cg * 8 + 2 * q] = acc[rr][q].x;
+          s_part[(slice * G + rr) * kModTmaCols + cg * 8 + 2 * q + 1] = acc[rr][q].y;
         }
     }
     __syncthreads();
@@ -271,7 +286,7 @@ modulation_tma_kernel(const __grid_constant__ CUtensorMap tmW, const ModParams p
       if (col_base + cc < p.N6) {
         float v = 0.f;
 #pragma unroll
-        for (int sl = 0; sl < kModTmaSlices; ++sl) v += s_part[(sl * kModReqGroup + rr) * kModTmaCols + cc];
+        for (int sl = 0; sl < kModTmaSlices; ++sl) v += s_part[(sl * G + rr) * kModTmaCols + cc];
         p.mod[(static_cast<size_t>(r0 + rr) * p.NB + blk) * p.N6 + col_base + cc] = v + bias[col_base + cc];
       }
     }
