@@ -50,7 +50,11 @@ struct AttnCfg {
   static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
   static constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;
   static constexpr int OFF_BAR = OFF_V + KV_STAGES * TILE_BYTES;
-  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+  // Every CTA takes all 512 tensor-memory columns, so two CTAs on one SM would only queue in tcgen05.alloc:
+  // the request is padded past half of the SM's shared memory so that exactly one CTA is resident (matters for
+  // head_dim 64, whose tiles alone need under 100 KB).
+  static constexpr int SMEM_USED = OFF_BAR + 256 + 1024;
+  static constexpr int SMEM_BYTES = SMEM_USED > 116 * 1024 ? SMEM_USED : 116 * 1024;
   static constexpr int THREADS = 384;
   static constexpr int Q_ROWS = 256;             // query rows per CTA
 };

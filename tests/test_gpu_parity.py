@@ -2,7 +2,18 @@
 
 Bar (per request): max|gpu - oracle| / rms(oracle) <= 1e-2 on the step output.
 Integer results and packed-vs-alone GPU outputs must be bit-identical.
+
+Every run of the helper below first fills the activation regions of the workspace with NaN bytes
+(`dit_debug_poison`), so a kernel that reads a row nobody wrote shows up as NaN in the output, and
+checks the guard areas between the regions afterwards (the stand-in for a memory checker).
+
+The long requests (1024^2 and 2048^2 through 4 and 8 blocks) are compared at full depth with oracle
+rows stored in tests/golden/deep_rows.npz (written by tests/golden/make_deep_rows.py from the oracle
+alone); for those the maximum runs over the stored rows and the rms is the oracle's over the whole
+request (also stored), and over the stored rows.
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -12,6 +23,23 @@ from paper_2510_01565_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 TOL = 1e-2   # max|gpu - oracle| / rms(oracle), per request
+
+DEEP_ROWS = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "deep_rows.npz")
+
+
+def check_deep_rows(run, out, cfg, r):
+    """Full-depth comparison of request r with the stored oracle rows of configuration `cfg`."""
+    with np.load(DEEP_ROWS) as z:
+        rows, ref = z[f"{cfg}/r{r}/rows"], z[f"{cfg}/r{r}/out"].astype(np.float64)
+        rms_full, rms_rows = float(z[f"{cfg}/r{r}/rms_full"]), float(z[f"{cfg}/r{r}/rms_rows"])
+        assert int(z[f"{cfg}/r{r}/n_tokens"]) == run.wl.token_lens[r] and int(z[f"{cfg}/r{r}/n_blocks"]) == run.nb
+    got = run.rows(out, r)[run.torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    dmax = float(np.abs(got - ref).max())
+    err_full, err_rows = dmax / rms_full, dmax / rms_rows
+    print(f"{cfg} request {r}: max|d|/rms over {len(rows)} stored rows = {err_full:.3e} (request rms), {err_rows:.3e} (rows' rms)")
+    assert err_full <= TOL and err_rows <= TOL, f"{cfg} request {r}: {err_full:.3e} / {err_rows:.3e}"
+    return err_full
 
 
 @pytest.fixture(scope="module")
@@ -52,18 +80,20 @@ class DeviceRun:
         self.cond = B.bits_to_cuda_bf16(wl.cond)
         self.cu = np.concatenate([[0], np.cumsum(wl.token_lens)])
 
-    def packed(self, n_blocks=None):
-        out = self.ctx.dit_step_forward(self.tok, self.wl.token_lens, self.cond, n_blocks or self.nb)
+    def _step(self, tok, lens, cond, n_blocks):
+        self.ctx.dit_debug_poison()                       # unwritten reads become NaN in the output
+        out = self.ctx.dit_step_forward(tok, lens, cond, n_blocks or self.nb)
         self.torch.cuda.synchronize()
         self.ctx.dit_ctx_poll_status()
+        assert self.ctx.dit_debug_check_guards() == 0, "a kernel wrote outside its region of the workspace"
         return out
+
+    def packed(self, n_blocks=None):
+        return self._step(self.tok, self.wl.token_lens, self.cond, n_blocks)
 
     def alone(self, r, n_blocks=None):
         a, b = int(self.cu[r]), int(self.cu[r + 1])
-        out = self.ctx.dit_step_forward(self.tok[a:b].contiguous(), [b - a], self.cond[r:r + 1].contiguous(), n_blocks or self.nb)
-        self.torch.cuda.synchronize()
-        self.ctx.dit_ctx_poll_status()
-        return out
+        return self._step(self.tok[a:b].contiguous(), [b - a], self.cond[r:r + 1].contiguous(), n_blocks)
 
     def rows(self, out, r):
         return out[int(self.cu[r]):int(self.cu[r + 1])]
@@ -130,8 +160,9 @@ def test_cfg3_1024_two_requests_packed(B):
     run = DeviceRun(B, wl)
     out = run.packed()
     check_packed_equals_alone(run, out)
-    # full 4-block oracle on the second request (it sits at a non-zero packed offset)
-    check_request(run, out, 1, oracle_requests(wl, [1])[1])
+    # both requests through all 4 blocks against the stored oracle rows
+    check_deep_rows(run, out, "cfg3_1024x2", 0)
+    check_deep_rows(run, out, "cfg3_1024x2", 1)
     run.close()
 
 
@@ -148,9 +179,10 @@ def test_cfg4_2048_long_sequence(B):
                           wl.dims.n_heads, wl.dims.ln_eps, rows=rows)
     got = out1.cpu().numpy().astype(np.float64)[rows]
     assert O.error_metric(got, ref) <= TOL
-    # the full 4-block step: finite, reproducible bit for bit
+    # the full 4-block step: finite, against the stored oracle rows, reproducible bit for bit
     out = run.packed()
     assert bool(run.torch.isfinite(out).all())
+    check_deep_rows(run, out, "cfg4_2048", 0)
     assert run.torch.equal(out, run.packed())
     run.close()
 
@@ -166,6 +198,9 @@ def test_cfg5_mixed_resolution_eight_requests(B):
     ref = oracle_requests(wl, [1, 2, 3])
     for r in (1, 2, 3):
         check_request(run, out, r, ref[r])
+    # a 1024^2 request and the 2048^2 request through all 8 blocks against the stored oracle rows
+    check_deep_rows(run, out, "cfg5_mixed8", 0)
+    check_deep_rows(run, out, "cfg5_mixed8", 5)
     # the 2048^2 request inside the packed batch, first block, sampled rows
     out1 = run.packed(n_blocks=1)
     r = 5
@@ -332,6 +367,52 @@ def test_error_codes(B):
     assert float(out.min()) == 7.0
     ctx.dit_ctx_poll_status()
     ctx.close()
+
+
+def test_bounded_wait_expiry_sets_the_status_word_once(B):
+    """The failure path of every kernel: a bounded wait that runs out makes the kernel return and set
+    the device status word.  A one-CTA test kernel waits (limit: tens of microseconds) on a barrier that
+    nothing signals; the poll then reports the timeout once and the context keeps working."""
+    wl = W.make_custom("expire", W.SMALL, 1, [(64, 64, 3)], seed=14, timestep_cond=False)
+    run = DeviceRun(B, wl)
+    want = run.packed()
+    run.ctx.dit_ctx_poll_status()                      # clean before
+    run.ctx.dit_debug_expire_wait()
+    run.torch.cuda.synchronize()
+    with pytest.raises(B.DitError) as e:
+        run.ctx.dit_ctx_poll_status()
+    assert e.value.status == 7 and "wait-expiry test" in str(e.value)      # DIT_ERR_TIMEOUT, names the kernel
+    run.ctx.dit_ctx_poll_status()                      # reported once, then clear
+    assert run.torch.equal(run.packed(), want)         # the context is still usable
+    run.close()
+
+
+def test_poison_hook_makes_unwritten_reads_visible(B):
+    """The poison fill itself: after it every activation tap reads as NaN and the guards are whole;
+    damaging a guard by hand is reported."""
+    import torch
+    wl = W.make_custom("poison", W.SMALL, 1, [(64, 64, 3)], seed=15, timestep_cond=False)
+    run = DeviceRun(B, wl)
+    run.packed()
+    run.ctx.dit_debug_poison()
+    torch.cuda.synchronize()
+    for name in ("h", "qkv", "attn", "u", "mod", "stream"):
+        assert bool(torch.isnan(run.ctx.dit_debug_tap(name).float()).all()), name
+    assert run.ctx.dit_debug_check_guards() == 0
+    # the guard right after the residual stream region: clobber one word through a view of the workspace
+    base = (run.ctx.workspace.data_ptr() + 1023) // 1024 * 1024 - run.ctx.workspace.data_ptr()
+    import ctypes as C
+    ptr, rows, cols, eb = C.c_void_p(), C.c_int64(), C.c_int64(), C.c_int32()
+    assert run.ctx.lib.dit_debug_tap(run.ctx.handle, B.TAPS["h"], C.byref(ptr), C.byref(rows), C.byref(cols), C.byref(eb)) == 0
+    h_off = ptr.value - run.ctx.workspace.data_ptr()
+    assert h_off - 1024 >= base
+    run.ctx.workspace[h_off - 1024:h_off - 1020] = 0           # last KiB before `h` is the stream's guard
+    assert run.ctx.dit_debug_check_guards() == 1
+    run.ctx.dit_debug_poison()                                 # rewrites the guards
+    assert run.ctx.dit_debug_check_guards() == 0
+    out = run.packed()
+    assert bool(torch.isfinite(out).all())
+    run.close()
 
 
 def test_step_replays_from_a_cuda_graph(B):
