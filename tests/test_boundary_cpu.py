@@ -77,7 +77,9 @@ def test_workspace_bytes_and_config_validation(lib):
                 dict(flags=8 | 1), dict(flags=8 | 2), dict(flags=8 | 4),     # bf16 operands: plain blocks only
                 dict(ln_eps=-1.0)]:
         assert ws(**bad) == 0, bad
-    assert ws(flags=7) == full        # the variant bits are accepted and cost no workspace
+    assert ws(flags=3) == full        # the QK variant bits are accepted and cost no workspace
+    # the e4m3 mode adds the quantised copy [T, H + F] of the tile-produced operands and their row scales
+    assert 9216 * (3072 + 12288) <= ws(flags=7) - full <= 9216 * (3072 + 12288) + 9216 * 4 + 4096
     assert ws(flags=8) == full        # so is the bf16-operand mode (same element sizes)
     assert lib.dit_workspace_bytes(None) == 0
 
