@@ -254,10 +254,21 @@ const RowGeom kNoGeom{};
 template <int EPI, int HD = 0, bool DUAL = false, bool FP8 = false, bool BF16 = false>
 cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                         const SeqInfo& seq, cudaStream_t st, const RowGeom& geo = kNoGeom, const CUtensorMap* tmB2 = nullptr) {
-  // Row band of the tile order: as many 256-row tiles of A as fit in about 36 MB of L2
+  // Band of the tile order: as many 256-row panels of one operand as fit in about 38 MB of L2 are held there
+  // while the other operand streams past.  Holding A costs A + W * (row bands) bytes of DRAM reads, holding the
+  // weights W + A * (column bands); the cheaper one is taken (long batches: the weights stay, the rows stream).
   GemmParams q = p;
-  const long long band_bytes = 2ll * gemm_cfg::BM * p.K * (FP8 ? 1 : 2);
-  q.band = static_cast<int>(std::max(1ll, std::min<long long>((36ll << 20) / band_bytes, (p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM))));
+  {
+    const long long esz = FP8 ? 1 : 2;
+    const long long panel = 2ll * gemm_cfg::BM * p.K * esz;                 // one 256-row panel of either operand
+    const long long num_m = (p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM), num_n = (p.N + gemm_cfg::BN - 1) / gemm_cfg::BN;
+    const long long fit = std::max(1ll, (38ll << 20) / panel);
+    const long long rb = std::min(fit, num_m), cb = std::min(fit, num_n);
+    const long long a_bytes = num_m * panel, w_bytes = num_n * panel;
+    const long long cost_rows = a_bytes + w_bytes * ((num_m + rb - 1) / rb);
+    const long long cost_cols = w_bytes + a_bytes * ((num_n + cb - 1) / cb);
+    q.band = (!DUAL && cost_cols < cost_rows) ? -static_cast<int>(cb) : static_cast<int>(rb);
+  }
   // 256 x 256 tiles, one per CTA pair; persistent grid of as many pairs as can be resident
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);   // a two-stream launch may have more items than row tiles: the loop covers them

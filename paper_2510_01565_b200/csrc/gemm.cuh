@@ -31,7 +31,7 @@ enum GemmEpilogue : int { kEpiBiasF16 = 0, kEpiBiasGeluF16 = 1, kEpiGateResidF32
 
 struct GemmParams {
   int M, N, K;
-  int band;                 // row tiles (of 256 rows) per band of the tile order, >= 1
+  int band;                 // > 0: row tiles (of 256 rows) per band of the tile order; < 0: column tiles per band
   const float* bias;        // [N]
   __half* out16;            // [M, N] with row stride ld16 elements (0 = N)
   const float* resid;       // [M, N]
@@ -91,16 +91,26 @@ __device__ __forceinline__ float2 gelu_tanh_f32x2(float2 z) {
   return ffma2(hz, t, hz);
 }
 
-// Tile order.  Row tiles are grouped in bands of `band`; inside a band the row index runs fastest and
-// every column tile is visited before the next band starts.  The tiles in flight then share one
-// band of A (sized by the host to stay in L2) while the weight tiles stream past, each read from
-// DRAM once per band.
+// Tile order.  band > 0: row tiles are grouped in bands of `band`; inside a band the row index runs fastest and
+// every column tile is visited before the next band starts.  The tiles in flight then share one band of A (sized
+// by the host to stay in L2) while the weight tiles stream past, each read from DRAM once per band.
+// band < 0: the same with the roles swapped: column tiles in bands of -band whose weight tiles stay in L2 while
+// the rows of A stream past, each read once per band.  The host picks whichever reads less from DRAM.
 __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int band, int& mb, int& nb) {
-  const int per_band = band * num_n;
-  const int b = t / per_band, r = t - b * per_band;
-  const int rows = min(band, num_m - b * band);               // the last band may be shorter
-  nb = r / rows;
-  mb = b * band + (r - nb * rows);
+  if (band > 0) {
+    const int per_band = band * num_n;
+    const int b = t / per_band, r = t - b * per_band;
+    const int rows = min(band, num_m - b * band);               // the last band may be shorter
+    nb = r / rows;
+    mb = b * band + (r - nb * rows);
+  } else {
+    const int cb = -band;
+    const int per_band = cb * num_m;
+    const int b = t / per_band, r = t - b * per_band;
+    const int cols = min(cb, num_n - b * cb);
+    mb = r / cols;
+    nb = b * cb + (r - mb * cols);
+  }
 }
 
 // DUAL: two-stream launch.  The weight operand comes from tmB for image-token rows and from tmB2 for
