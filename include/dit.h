@@ -208,11 +208,26 @@ dit_status dit_step_forward_requests(dit_ctx *ctx, const void *packed_tokens, co
  * step where the data flow allows it: the tokens go in as four row slices on a copy stream of the
  * context and block 0 normalises and projects each slice as it lands; the part of the last block that
  * follows attention runs in the same row slices (only its last GEMM for parallel blocks and in the
- * e4m3 mode) and every finished slice of `out` goes back while the next one computes.  The results are
+ * e4m3 mode) and every finished slice of `out` goes back, on a stream of its own, while the next one computes.  The results are
  * those of dit_step_forward bit for bit.  Use pinned host memory (pageable memory serialises the copies). */
 dit_status dit_step_forward_host(dit_ctx *ctx, const void *host_packed_tokens,
                                  const int32_t *per_request_token_lens, int32_t n_requests,
                                  const void *host_cond, int32_t n_blocks, float *host_out, void *stream);
+
+/* The same step without the final wait, for a serving loop that keeps two steps in flight (the paper's workers
+ * run step after step of their round, Section 5.2): the call returns once everything is enqueued, and
+ * dit_host_wait(ctx, calls_back) blocks until the output of the latest such call (calls_back = 0) or of the one
+ * before it (calls_back = 1) has arrived in its host buffer.  Successive calls on one context overlap where the
+ * data allow: the tokens of call k + 1 go in as soon as block 0 of call k has read the staging buffer, and the
+ * output of call k goes out while call k + 1 computes (the step itself waits for that copy before it overwrites
+ * the device-side output).  Rules: issue the calls of one context on one stream; keep host_packed_tokens,
+ * host_cond and host_out of a call untouched until dit_host_wait has covered it; at most two calls may be
+ * outstanding (wait for call k - 1 before issuing call k + 1); an empty batch (n_requests == 0) does not count as
+ * a call.  dit_step_forward_host is this call followed by dit_host_wait(ctx, 0). */
+dit_status dit_step_forward_host_async(dit_ctx *ctx, const void *host_packed_tokens,
+                                       const int32_t *per_request_token_lens, int32_t n_requests,
+                                       const void *host_cond, int32_t n_blocks, float *host_out, void *stream);
+dit_status dit_host_wait(dit_ctx *ctx, int32_t calls_back);
 
 /* Reads (with a device synchronisation) the device status word that kernels set when a bounded wait
  * runs out; returns DIT_OK or DIT_ERR_TIMEOUT and clears the word. */

@@ -26,7 +26,7 @@ KERNEL_KINDS = ["modulation", "ln_modulate", "gemm_qkv", "attention", "gemm_proj
 TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights", "dit_load_dual_block_weights",
-           "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host",
+           "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host", "dit_step_forward_host_async", "dit_host_wait",
            "dit_ctx_poll_status", "dit_debug_tap", "dit_debug_poison", "dit_debug_check_guards", "dit_debug_expire_wait", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
            "dit_denoise_step", "dit_denoise_round", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
@@ -111,6 +111,10 @@ def load_library() -> C.CDLL:
     lib.dit_step_forward.argtypes = [vp, vp, C.POINTER(i32), i32, vp, i32, vp, vp]
     lib.dit_step_forward_host.restype = C.c_int
     lib.dit_step_forward_host.argtypes = [vp, vp, C.POINTER(i32), i32, vp, i32, vp, vp]
+    lib.dit_step_forward_host_async.restype = C.c_int
+    lib.dit_step_forward_host_async.argtypes = [vp, vp, C.POINTER(i32), i32, vp, i32, vp, vp]
+    lib.dit_host_wait.restype = C.c_int
+    lib.dit_host_wait.argtypes = [vp, i32]
     lib.dit_ctx_poll_status.restype = C.c_int
     lib.dit_ctx_poll_status.argtypes = [vp]
     lib.dit_debug_tap.restype = C.c_int
@@ -370,6 +374,21 @@ class DitContext:
                                                    C.c_void_p(host_cond.data_ptr()), n_blocks,
                                                    C.c_void_p(host_out.data_ptr()), self._stream(stream)))
         return host_out
+
+    def dit_step_forward_host_async(self, host_tokens, token_lens, host_cond, n_blocks: int, host_out, stream=None):
+        """The same without the final wait; dit_host_wait(0 or 1) covers the latest call or the one before."""
+        lens = self._lens(token_lens)
+        assert not host_tokens.is_cuda and not host_cond.is_cuda and not host_out.is_cuda
+        assert host_tokens.is_contiguous() and host_cond.is_contiguous() and host_out.is_contiguous()
+        assert host_tokens.shape == (int(lens.sum()), self.hidden) and host_out.shape == host_tokens.shape
+        self._check(self.lib.dit_step_forward_host_async(self.handle, C.c_void_p(host_tokens.data_ptr()),
+                                                         lens.ctypes.data_as(C.POINTER(C.c_int32)), len(lens),
+                                                         C.c_void_p(host_cond.data_ptr()), n_blocks,
+                                                         C.c_void_p(host_out.data_ptr()), self._stream(stream)))
+        return host_out
+
+    def dit_host_wait(self, calls_back: int = 0):
+        self._check(self.lib.dit_host_wait(self.handle, calls_back))
 
     # ------------------------------------------------------------------ shell around the block stack
     @staticmethod

@@ -180,8 +180,14 @@ struct dit_ctx {
   // optional per-kernel timing (CUDA events recorded around every launch of a step)
   bool timing;
   // dit_step_forward_host: the output goes back to the host in row slices while the last GEMM still runs
-  cudaStream_t copy_stream;
-  cudaEvent_t slice_done[kHostOutSlices], copies_done, tok_ready[kHostOutSlices];
+  cudaStream_t copy_stream;                // device -> host copies of the output slices
+  cudaStream_t h2d_stream;                 // host -> device copies of the token slices (the link is full duplex)
+  cudaEvent_t slice_done[kHostOutSlices], tok_ready[kHostOutSlices];
+  cudaEvent_t tok_consumed;                // block 0 of the last host-buffer step has read the staging tokens
+  cudaEvent_t st_entry;                    // everything enqueued on the caller's stream before a host-buffer call
+  bool last_step_from_host;                // the last step on this context was a host-buffer step
+  cudaEvent_t d2h_done[2];                 // output of host-buffer call c has arrived: d2h_done[c & 1]
+  uint64_t host_calls;                     // host-buffer calls so far
   bool host_copied;                        // the last step_impl call sent its output to the host itself
   std::vector<cudaEvent_t> ev_pool;        // pairs: [2i] start, [2i+1] stop
   std::vector<int> ev_kind;                // kind of pair i
@@ -449,6 +455,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     }
     const int tile_rows = 2 * gemm_cfg::BM;
     const int per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;   // rows per slice
+    // the previous host-buffer call may still be copying its output out of the same device buffer
+    DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->d2h_done[(ctx->host_calls & 1) ^ 1], 0));
     for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
       const int rows = std::min(per, T - r0);
       CUtensorMap tmA;
@@ -466,7 +474,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out + static_cast<size_t>(r0) * g.N, g.out32 + static_cast<size_t>(r0) * g.N,
                                         static_cast<size_t>(rows) * g.N * 4, cudaMemcpyDeviceToHost, ctx->copy_stream));
     }
-    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, ctx->copy_stream));
+    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->d2h_done[ctx->host_calls & 1], ctx->copy_stream));
     ctx->host_copied = true;
     return DIT_OK;
   };
@@ -591,6 +599,10 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       const dit_status ls = ln1_qkv(0, T, tm_h);
       if (ls != DIT_OK) return ls;
     }
+    // the packed tokens are read by block 0's LayerNorm only: from here on the staging buffer may be refilled for
+    // the next host-buffer step (recorded for those steps only: they are never part of a stream capture, and an
+    // event recorded inside a capture could not be waited for outside it)
+    if (b == 0 && host_out) DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->tok_consumed, st));
     // attention (one pass over all tokens of a request, whatever their stream)
     AttnParams ap{};
     ap.out = bs.parallel ? cat : a; ap.ld_out = bs.parallel ? H + F : H;
@@ -642,6 +654,8 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
       // exactly as in the unsliced launches.
       const int tile_rows = 2 * gemm_cfg::BM;
       const int per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;
+      // the previous host-buffer call may still be copying its output out of the same device buffer
+      DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->d2h_done[(ctx->host_calls & 1) ^ 1], 0));
       for (int sidx = 0, r0 = 0; r0 < T; ++sidx, r0 += per) {
         const int rows = std::min(per, T - r0);
         const size_t eH = static_cast<size_t>(r0) * H, eF = static_cast<size_t>(r0) * F;
@@ -680,7 +694,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
         DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->slice_done[sidx], 0));
         DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out + eH, out + eH, static_cast<size_t>(rows) * H * 4, cudaMemcpyDeviceToHost, ctx->copy_stream));
       }
-      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, ctx->copy_stream));
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->d2h_done[ctx->host_calls & 1], ctx->copy_stream));
       ctx->host_copied = true;
       continue;
     }
@@ -747,6 +761,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   ctx->last_launches = launches;
   ctx->last_T = T; ctx->last_R = n; ctx->last_nb = n_blocks;
   ctx->last_parallel = ctx->blocks[n_blocks - 1].parallel;
+  ctx->last_step_from_host = host_out != nullptr;
   return DIT_OK;
 }
 
@@ -883,8 +898,13 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
     ctx->gemm_pairs = std::max(1, std::min(clusters, sms / 2));
   }
   ctx->copy_stream = nullptr;
+  ctx->h2d_stream = nullptr;
   ctx->host_copied = false;
-  ctx->copies_done = nullptr;
+  ctx->host_calls = 0;
+  ctx->tok_consumed = nullptr;
+  ctx->st_entry = nullptr;
+  ctx->last_step_from_host = false;
+  ctx->d2h_done[0] = ctx->d2h_done[1] = nullptr;
   for (int i = 0; i < kHostOutSlices; ++i) { ctx->slice_done[i] = nullptr; ctx->tok_ready[i] = nullptr; }
   {
     const cuuint64_t dims[3] = {static_cast<cuuint64_t>(6) * cfg->hidden, static_cast<cuuint64_t>(cfg->cond_dim), static_cast<cuuint64_t>(cfg->max_blocks)};
@@ -896,9 +916,12 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
   }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->tok_consumed, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->st_entry, cudaEventDisableTiming);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->d2h_done[i], cudaEventDisableTiming);
   for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->slice_done[i], cudaEventDisableTiming);
   for (int i = 0; i < kHostOutSlices && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->tok_ready[i], cudaEventDisableTiming);
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->copies_done, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(ctx->ws + lay.status, 0, 256);
   for (int g = 0; g < lay.n_guards && e == cudaSuccess; ++g) {
     fill_u32_kernel<<<1, 256>>>(reinterpret_cast<uint32_t*>(ctx->ws + lay.guard[g]), kGuardPattern, static_cast<int>(kGuardBytes / 4));
@@ -921,8 +944,11 @@ dit_status dit_ctx_destroy(dit_ctx* ctx) {
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   for (int i = 0; i < kHostOutSlices; ++i) if (ctx->slice_done[i]) cudaEventDestroy(ctx->slice_done[i]);
   for (int i = 0; i < kHostOutSlices; ++i) if (ctx->tok_ready[i]) cudaEventDestroy(ctx->tok_ready[i]);
-  if (ctx->copies_done) cudaEventDestroy(ctx->copies_done);
+  if (ctx->tok_consumed) cudaEventDestroy(ctx->tok_consumed);
+  if (ctx->st_entry) cudaEventDestroy(ctx->st_entry);
+  for (int i = 0; i < 2; ++i) if (ctx->d2h_done[i]) cudaEventDestroy(ctx->d2h_done[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
   delete[] ctx->blocks;
   delete ctx;
   return DIT_OK;
@@ -1116,10 +1142,10 @@ dit_status dit_step_forward(dit_ctx* ctx, const void* packed_tokens, const int32
   return step_impl(ctx, packed_tokens, lens, n, cond, n_blocks, out, static_cast<cudaStream_t>(stream));
 }
 
-dit_status dit_step_forward_host(dit_ctx* ctx, const void* host_tokens, const int32_t* lens, int32_t n,
-                                 const void* host_cond, int32_t n_blocks, float* host_out, void* stream) {
+dit_status dit_step_forward_host_async(dit_ctx* ctx, const void* host_tokens, const int32_t* lens, int32_t n,
+                                       const void* host_cond, int32_t n_blocks, float* host_out, void* stream) {
   dit_status s = check_step_args(ctx, host_tokens, lens, n, host_cond, n_blocks, host_out);
-  if (s != DIT_OK || n == 0) return s;
+  if (s != DIT_OK || n == 0) return s;            // an empty batch is a no-op and does not count as a call
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   size_t T = 0;
   for (int r = 0; r < n; ++r) T += lens[r];
@@ -1127,31 +1153,58 @@ dit_status dit_step_forward_host(dit_ctx* ctx, const void* host_tokens, const in
   void* d_tok = ctx->ws + ctx->lay.stage_tokens;
   void* d_cond = ctx->ws + ctx->lay.stage_cond;
   float* d_out = ctx->at<float>(ctx->lay.stage_out);
-  // cond first (the modulation kernel needs nothing else), then the tokens in row slices on the copy stream:
-  // block 0 starts on a slice as soon as it has landed, the slices behind it overlap its work
+  // cond first (the modulation kernel needs nothing else; it follows the previous step on `st`), then the
+  // tokens in row slices on the host-to-device stream: they may go in as soon as block 0 of the PREVIOUS step
+  // has read the staging buffer, i.e. under that step's remaining blocks; block 0 of this step starts on a
+  // slice as soon as it has landed
   DIT_CUDA_TRY(ctx, cudaMemcpyAsync(d_cond, host_cond, n * C * 2, cudaMemcpyHostToDevice, st));
   {
-    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->copies_done, st));                 // order the copy stream after earlier work on st
-    DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->copies_done, 0));
+    if (ctx->last_step_from_host) {
+      DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->h2d_stream, ctx->tok_consumed, 0));
+    } else {
+      // some other step (or a replayed graph of one) may still be reading the staging buffer: wait for all of it
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->st_entry, st));
+      DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->h2d_stream, ctx->st_entry, 0));
+    }
     const size_t tile_rows = 2 * gemm_cfg::BM;
     const size_t per = ((T + tile_rows - 1) / tile_rows + kHostOutSlices - 1) / kHostOutSlices * tile_rows;
     for (size_t sidx = 0, r0 = 0; sidx < static_cast<size_t>(kHostOutSlices); ++sidx, r0 += per) {
       if (r0 < T) {
         const size_t rows = std::min(per, T - r0);
         DIT_CUDA_TRY(ctx, cudaMemcpyAsync(static_cast<uint8_t*>(d_tok) + r0 * H * 2, static_cast<const uint8_t*>(host_tokens) + r0 * H * 2,
-                                          rows * H * 2, cudaMemcpyHostToDevice, ctx->copy_stream));
+                                          rows * H * 2, cudaMemcpyHostToDevice, ctx->h2d_stream));
       }
-      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->tok_ready[sidx], ctx->copy_stream));
+      DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->tok_ready[sidx], ctx->h2d_stream));
     }
   }
   ctx->host_copied = false;
+  const uint64_t call = ctx->host_calls;           // step_impl records this call's arrival event d2h_done[call & 1]
   s = step_impl(ctx, d_tok, lens, n, d_cond, n_blocks, d_out, st, nullptr, host_out, true);
   if (s != DIT_OK) return s;
-  // the output normally went back slice by slice on the copy stream (see step_impl): join it
-  if (ctx->host_copied) DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->copies_done, 0));
-  else DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, d_out, T * H * 4, cudaMemcpyDeviceToHost, st));
-  DIT_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  // the output normally goes back slice by slice on the copy stream (see step_impl); otherwise in one piece here
+  if (!ctx->host_copied) {
+    DIT_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->d2h_done[(call & 1) ^ 1], 0));
+    DIT_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, d_out, T * H * 4, cudaMemcpyDeviceToHost, st));
+    DIT_CUDA_TRY(ctx, cudaEventRecord(ctx->d2h_done[call & 1], st));
+  }
+  ctx->host_calls = call + 1;
   return DIT_OK;
+}
+
+dit_status dit_host_wait(dit_ctx* ctx, int32_t calls_back) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (calls_back < 0 || calls_back > 1) return fail(ctx, DIT_ERR_INVALID_ARG, "calls_back must be 0 (the latest call) or 1 (the one before)");
+  if (ctx->host_calls <= static_cast<uint64_t>(calls_back)) return DIT_OK;        // no such call yet
+  DIT_CUDA_TRY(ctx, cudaEventSynchronize(ctx->d2h_done[(ctx->host_calls - 1 - calls_back) & 1]));
+  return DIT_OK;
+}
+
+dit_status dit_step_forward_host(dit_ctx* ctx, const void* host_tokens, const int32_t* lens, int32_t n,
+                                 const void* host_cond, int32_t n_blocks, float* host_out, void* stream) {
+  const dit_status s = dit_step_forward_host_async(ctx, host_tokens, lens, n, host_cond, n_blocks, host_out, stream);
+  if (s != DIT_OK || n == 0) return s;
+  return dit_host_wait(ctx, 0);
 }
 
 dit_status dit_ctx_poll_status(dit_ctx* ctx) {

@@ -213,6 +213,23 @@ def test_cfg5_mixed_resolution_eight_requests(B):
     run.close()
 
 
+def test_cfg5_another_seeded_mix(B):
+    """The mixed-resolution configuration drawn with another seed (another resolution mix, request order and
+    set of packed offsets: 512, 512, 1024, 256, 1024, 1024, 256, 256): the last 512^2 and the last 256^2 request
+    against the oracle through all 8 blocks, everything finite, packed == alone for one request of each
+    resolution present."""
+    wl = W.make_workload("cfg5_mixed8", seed=2)
+    assert [q.height for q in wl.requests] == [512, 512, 1024, 256, 1024, 1024, 256, 256]
+    run = DeviceRun(B, wl)
+    out = run.packed()
+    assert bool(run.torch.isfinite(out).all())
+    ref = oracle_requests(wl, [1, 7])
+    check_request(run, out, 1, ref[1])
+    check_request(run, out, 7, ref[7])
+    check_packed_equals_alone(run, out, requests=[1, 4, 7])
+    run.close()
+
+
 # ----------------------------------------------------------------------------- edge cases
 @pytest.mark.parametrize("dims,reqs", [
     (W.LARGE, [(16, 16, 0)]),                                    # a single token: a = v
@@ -332,6 +349,42 @@ def test_pack_tokens_and_host_entry_point(B):
     h_out = torch.empty(out.shape, dtype=torch.float32).pin_memory()
     run.ctx.dit_step_forward_host(h_tok, wl.token_lens, h_cond, 1, h_out)
     assert torch.equal(h_out, out.cpu())
+    run.close()
+
+
+def test_host_steps_two_in_flight(B):
+    """dit_step_forward_host_async keeps two steps in flight: the tokens of step k + 1 go in under step k and
+    the output of step k goes out under step k + 1.  Six steps alternate two different batches of the same shape
+    through two host output buffers; every delivered output is bit-identical to the device-buffer step of its
+    batch, whatever the copies overlapped with."""
+    import torch
+    wl_a = W.make_custom("pipe_a", W.LARGE, 2, [(512, 512, 96), (256, 256, 64)], seed=31)
+    wl_b = W.make_custom("pipe_b", W.LARGE, 2, [(512, 512, 96), (256, 256, 64)], seed=32)
+    run = DeviceRun(B, wl_a)                                   # both batches run on wl_a's weights
+    want = []
+    for wl in (wl_a, wl_b):
+        out = run.ctx.dit_step_forward(B.bits_to_cuda_bf16(wl.packed_tokens()), wl.token_lens, B.bits_to_cuda_bf16(wl.cond), 2)
+        torch.cuda.synchronize()
+        want.append(out.cpu())
+    assert not torch.equal(want[0], want[1])
+    h_tok = [torch.from_numpy(wl.packed_tokens().view(np.int16)).pin_memory() for wl in (wl_a, wl_b)]
+    h_cond = [torch.from_numpy(wl.cond.view(np.int16)).pin_memory() for wl in (wl_a, wl_b)]
+    h_out = [torch.full(want[0].shape, float("nan"), dtype=torch.float32).pin_memory() for _ in range(2)]
+    lens = wl_a.token_lens
+    ctx = run.ctx
+    ctx.dit_host_wait(0)                                       # nothing outstanding yet: returns at once
+    ctx.dit_step_forward_host_async(h_tok[0], lens, h_cond[0], 2, h_out[0])
+    for k in range(1, 6):
+        ctx.dit_step_forward_host_async(h_tok[k & 1], lens, h_cond[k & 1], 2, h_out[k & 1])
+        ctx.dit_host_wait(1)                                   # step k - 1 has arrived
+        assert torch.equal(h_out[(k - 1) & 1], want[(k - 1) & 1]), f"step {k - 1}"
+        h_out[(k - 1) & 1].fill_(float("nan"))                 # its buffer is free again for step k + 1
+    ctx.dit_host_wait(0)
+    assert torch.equal(h_out[1], want[1])
+    with pytest.raises(B.DitError) as e:
+        ctx.dit_host_wait(2)
+    assert e.value.status == 1
+    ctx.dit_ctx_poll_status()
     run.close()
 
 
