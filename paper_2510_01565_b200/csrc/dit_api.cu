@@ -161,6 +161,9 @@ struct BlockState {
 
 constexpr int kHostOutSlices = 4;
 
+// Tensor maps of the activation buffers for one batch length T (a8, u8, cat8: the e4m3 mode's quantised copies).
+struct ActMaps { CUtensorMap h, a, u, qkv, cat, a8, u8, cat8; };
+
 struct dit_ctx {
   dit_config cfg;
   Layout lay;
@@ -173,6 +176,8 @@ struct dit_ctx {
   CUtensorMap tm_wout;                     // W_out^T, fp16 [kWoutRows, H]
   CUtensorMap tm_wada;                     // every block's W_ada as one 3-D tensor [max_blocks, C, 6H] bf16, boxes of 10 x 256
   bool tm_wada_ok;
+  ActMaps maps;                            // valid for batch length maps_T (-1: none yet)
+  int maps_T;
   int64_t last_launches;
   int last_T, last_R, last_nb;
   bool last_parallel;                      // the last block of the last step was a parallel block
@@ -396,22 +401,28 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
   // a parallel block writes attention and MLP outputs side by side into one [T, H + F] buffer that
   // starts where `a` starts and runs on into `u` (the two regions are consecutive)
   __half* cat = a;
-  CUtensorMap tm_h, tm_a, tm_u, tm_qkv, tm_cat;
-  if (!make_map(ctx, &tm_h, h, H, T, gemm_cfg::BM) || !make_map(ctx, &tm_a, a, H, T, gemm_cfg::BM) ||
-      !make_map(ctx, &tm_u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &tm_qkv, qkv, 3 * H, T, 128) ||
-      !make_map(ctx, &tm_cat, cat, H + F, T, gemm_cfg::BM))
-    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  // The activation tensor maps depend on the workspace (fixed) and on T only: they are encoded when T changes and
+  // kept in the context (a serving loop repeats the same batch shape for every step of a round).
   float* row_scale = ctx->at<float>(ctx->lay.row_scale);
-  if (fp8 && !make_map8(ctx, &tm_h, h, H, T, gemm_cfg::BM))   // h holds e4m3 codes in this mode
-    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   // e4m3 mode: the operands that are produced tile by tile (attention output, GELU output, or the two side by
   // side in a parallel block) are quantised row by row into q8 by a pass of their own before the GEMM that reads them
   uint8_t* q8 = ctx->at<uint8_t>(ctx->lay.q8);
   float* row_scale2 = ctx->at<float>(ctx->lay.row_scale2);
-  CUtensorMap tm_a8, tm_u8, tm_cat8;
-  if (fp8 && (!make_map8(ctx, &tm_a8, q8, H, T, gemm_cfg::BM) || !make_map8(ctx, &tm_u8, q8, F, T, gemm_cfg::BM) ||
-              !make_map8(ctx, &tm_cat8, q8, H + F, T, gemm_cfg::BM)))
-    return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  if (ctx->maps_T != T) {
+    ActMaps& m = ctx->maps;
+    ctx->maps_T = -1;
+    if (!make_map(ctx, &m.h, h, H, T, gemm_cfg::BM) || !make_map(ctx, &m.a, a, H, T, gemm_cfg::BM) ||
+        !make_map(ctx, &m.u, u, F, T, gemm_cfg::BM) || !make_map(ctx, &m.qkv, qkv, 3 * H, T, 128) ||
+        !make_map(ctx, &m.cat, cat, H + F, T, gemm_cfg::BM))
+      return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+    if (fp8 && (!make_map8(ctx, &m.h, h, H, T, gemm_cfg::BM) ||       // h holds e4m3 codes in this mode
+                !make_map8(ctx, &m.a8, q8, H, T, gemm_cfg::BM) || !make_map8(ctx, &m.u8, q8, F, T, gemm_cfg::BM) ||
+                !make_map8(ctx, &m.cat8, q8, H + F, T, gemm_cfg::BM)))
+      return fail(ctx, DIT_ERR_CUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+    ctx->maps_T = T;
+  }
+  const CUtensorMap &tm_h = ctx->maps.h, &tm_a = ctx->maps.a, &tm_u = ctx->maps.u, &tm_qkv = ctx->maps.qkv, &tm_cat = ctx->maps.cat;
+  const CUtensorMap &tm_a8 = ctx->maps.a8, &tm_u8 = ctx->maps.u8, &tm_cat8 = ctx->maps.cat8;
   auto quantise_rows = [&](const __half* src, long long ld, int K) -> cudaError_t {
     quantize_rows_e4m3_kernel<<<(T + kQuantWarps - 1) / kQuantWarps, kQuantWarps * 32, 0, st>>>(src, ld, q8, row_scale2, T, K);
     return cudaGetLastError();
@@ -836,6 +847,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->blocks = new (std::nothrow) BlockState[cfg->max_blocks];
   ctx->shell_loaded = false;
   ctx->last_launches = 0;
+  ctx->maps_T = -1;
   ctx->last_T = ctx->last_R = ctx->last_nb = 0;
   ctx->last_parallel = false;
   ctx->timing = false;
