@@ -38,6 +38,8 @@ struct AttnParams {
   int n_heads;
   float scale_log2;   // log2(e) / sqrt(d)
   int* status;
+  int* probe;         // test hook, NULL normally: [0] SM clock in MHz seen by a CTA of this launch (cycle counter
+                      // against the global nanosecond timer over the CTA's life), [1] its cycles per key block
 };
 
 template <int D>
@@ -90,6 +92,8 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  long long probe_c0 = 0; uint64_t probe_t0 = 0;
+  if (p.probe && threadIdx.x == 0) { probe_c0 = clock64(); probe_t0 = global_ns(); }
 
   // ---- which (request, head, 256-row query block) this CTA owns: requests longest first, and within a
   // request head-major, so that the CTAs resident at one time share the K/V of a few heads (a long
@@ -338,6 +342,12 @@ done:
   __syncthreads();
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
   if (threadIdx.x == 0 && *abort_flag) atomicMax(p.status, kStatusAttnTimeout);
+  if (p.probe && threadIdx.x == 0 && nkv >= 16) {      // long enough for the two timers to resolve the clock
+    const long long dc = clock64() - probe_c0;
+    const uint64_t dt = global_ns() - probe_t0;
+    p.probe[0] = static_cast<int>(dc * 1000 / static_cast<long long>(dt ? dt : 1));
+    p.probe[1] = static_cast<int>(dc / nkv);
+  }
 }
 
 }  // namespace dit

@@ -176,6 +176,7 @@ struct dit_ctx {
   CUtensorMap tm_wout;                     // W_out^T, fp16 [kWoutRows, H]
   CUtensorMap tm_wada;                     // every block's W_ada as one 3-D tensor [max_blocks, C, 6H] bf16, boxes of 10 x 256
   bool tm_wada_ok;
+  bool attn_probe;                         // test hook: attention CTAs record the SM clock they ran at
   ActMaps maps;                            // valid for batch length maps_T (-1: none yet)
   int maps_T;
   int64_t last_launches;
@@ -618,6 +619,7 @@ dit_status step_impl(dit_ctx* ctx, const void* tokens, const int32_t* lens, int 
     AttnParams ap{};
     ap.out = bs.parallel ? cat : a; ap.ld_out = bs.parallel ? H + F : H;
     ap.H = H; ap.n_heads = c.n_heads; ap.status = status;
+    ap.probe = ctx->attn_probe ? status + 4 : nullptr;
     ap.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c.head_dim));
     DIT_CUDA_TRY(ctx, timed(DIT_KERNEL_ATTENTION, [&] {
       if (bf) return c.head_dim == 128 ? launch_attention<128, true>(tm_qkv, ap, seq, st) : launch_attention<64, true>(tm_qkv, ap, seq, st);
@@ -848,6 +850,7 @@ dit_status dit_ctx_create(const dit_config* cfg, void* workspace, size_t workspa
   ctx->shell_loaded = false;
   ctx->last_launches = 0;
   ctx->maps_T = -1;
+  ctx->attn_probe = false;
   ctx->last_T = ctx->last_R = ctx->last_nb = 0;
   ctx->last_parallel = false;
   ctx->timing = false;
@@ -1273,6 +1276,19 @@ dit_status dit_debug_check_guards(dit_ctx* ctx, int32_t* n_damaged) {
     for (size_t i = 0; i < kGuardBytes / 4; ++i)
       if (host[i] != kGuardPattern) { ++*n_damaged; break; }
   }
+  return DIT_OK;
+}
+
+dit_status dit_debug_attention_probe(dit_ctx* ctx, int32_t enabled, int32_t* sm_mhz, int32_t* cycles_per_key_block) {
+  if (!ctx) return DIT_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  DIT_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  int word[2] = {0, 0};
+  DIT_CUDA_TRY(ctx, cudaMemcpy(word, ctx->at<int>(ctx->lay.status) + 4, sizeof(word), cudaMemcpyDeviceToHost));
+  DIT_CUDA_TRY(ctx, cudaMemset(ctx->at<int>(ctx->lay.status) + 4, 0, sizeof(word)));
+  if (sm_mhz) *sm_mhz = word[0];
+  if (cycles_per_key_block) *cycles_per_key_block = word[1];
+  ctx->attn_probe = enabled != 0;
   return DIT_OK;
 }
 
