@@ -212,7 +212,7 @@ class DeviceBench:
         sampler.start()
         if per_kernel:
             self.ctx.dit_ctx_set_timing(True)
-            self.ctx.dit_debug_attention_probe(True)     # the SM clock attention CTAs really run at inside the step
+            self.ctx.dit_debug_clock_probe(True)         # the SM clock attention and GEMM CTAs really run at inside the step
         self.barrier()
         self.e0.record(self.stream)
         for _ in range(n_steps):
@@ -225,7 +225,7 @@ class DeviceBench:
         if per_kernel:
             kernels = self.ctx.dit_ctx_read_timing()
             self.ctx.dit_ctx_set_timing(False)
-            self.attention_probe = self.ctx.dit_debug_attention_probe(False)
+            self.clock_probe = self.ctx.dit_debug_clock_probe(False)
         self.ctx.dit_ctx_poll_status()
         return ms, clocks, kernels
 
@@ -298,13 +298,17 @@ def step_summary(bench, ms_step, n_steps, clocks, kernels, peaks):
     roofline, roofline_attention = bench.rooflines(kern, kernels, flops, peaks)
     # attention against the chip's peak AT THE CLOCK ITS CTAs RAN AT (the part is power-capped and clocks kernels
     # differently; nvidia-smi's samples cannot be attributed to a kernel): SMs x 8192 dense fp16 FLOP per cycle x MHz
-    mhz, cyc = getattr(bench, "attention_probe", (0, 0))
+    mhz, cyc, gemm_mhz = getattr(bench, "clock_probe", (0, 0, 0))
+    sms = bench.torch.cuda.get_device_properties(bench.torch.cuda.current_device()).multi_processor_count
+    how = "clock64 against %globaltimer over one CTA's life (dit_debug_clock_probe)"
     if roofline_attention is not None and mhz > 0:
-        sms = bench.torch.cuda.get_device_properties(bench.torch.cuda.current_device()).multi_processor_count
         peak_at_clock = sms * 8192 * mhz * 1e6 / 1e12
         roofline_attention["in_kernel"] = {"sm_mhz": mhz, "cycles_per_key_block": cyc, "peak_at_that_clock_tflops": peak_at_clock,
-                                           "frac_of_peak_at_that_clock": roofline_attention["achieved"] / peak_at_clock,
-                                           "how": "clock64 against %globaltimer over one CTA's life (dit_debug_attention_probe)"}
+                                           "frac_of_peak_at_that_clock": roofline_attention["achieved"] / peak_at_clock, "how": how}
+    if gemm_mhz > 0:
+        peak_at_clock = sms * 8192 * gemm_mhz * 1e6 / 1e12
+        roofline["in_kernel"] = {"sm_mhz": gemm_mhz, "peak_at_that_clock_tflops": peak_at_clock,
+                                 "frac_of_peak_at_that_clock": roofline["achieved"] / peak_at_clock, "how": how}
     return {"workload": wl.name, "steps": n_steps, "ms_per_step": ms_step,
             "value": bench.replicas.whole_job_rate(wl.image_tokens, bench.world, ms_step), "unit": UNIT,
             "tflops": tflops,

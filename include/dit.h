@@ -251,13 +251,15 @@ dit_status dit_debug_tap(dit_ctx *ctx, dit_tap which, const void **ptr, int64_t 
 dit_status dit_debug_poison(dit_ctx *ctx, void *stream);
 dit_status dit_debug_check_guards(dit_ctx *ctx, int32_t *n_damaged);
 
-/* Measurement hook: while enabled, one thread of every attention CTA that sweeps at least 16 key blocks reads the
- * SM's cycle counter and the global nanosecond timer at its start and end and leaves (cycles * 1000 / ns, cycles per
- * key block) in the context's status area (last writer wins).  The call synchronises the device, returns the values
- * left since the previous call (0, 0 if none; either pointer may be NULL), clears them and sets the new state.
- * The step is power-capped, so the clock a kernel actually runs at inside a step (which a sampler outside the
- * process cannot attribute to a kernel) is what its tensor-pipe utilisation has to be read against. */
-dit_status dit_debug_attention_probe(dit_ctx *ctx, int32_t enabled, int32_t *sm_mhz, int32_t *cycles_per_key_block);
+/* Measurement hook: while enabled, one thread of every attention CTA that sweeps at least 16 key blocks, and of every
+ * GEMM CTA that lives 20 us or more, reads the SM's cycle counter and the global nanosecond timer at its start and end
+ * and leaves cycles * 1000 / ns (the SM clock in MHz it ran at; attention also its cycles per key block) in the
+ * context's status area (last writer wins).  The call synchronises the device, returns the values left since the
+ * previous call (0 if none; any pointer may be NULL), clears them and sets the new state.  The step is power-capped,
+ * so the clock a kernel actually runs at inside a step (which a sampler outside the process cannot attribute to a
+ * kernel) is what its tensor-pipe utilisation has to be read against. */
+dit_status dit_debug_clock_probe(dit_ctx *ctx, int32_t enabled, int32_t *attention_mhz, int32_t *cycles_per_key_block,
+                                 int32_t *gemm_mhz);
 
 /* Test hook for the failure path: launches one CTA that waits, with the library's bounded-wait
  * routine and a limit of about 50 microseconds, on a barrier that nothing ever signals.  The wait runs

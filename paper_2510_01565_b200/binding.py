@@ -27,7 +27,7 @@ TAPS = {"h": 0, "qkv": 1, "attn": 2, "u": 3, "mod": 4, "stream": 5}
 
 EXPORTS = ["dit_workspace_bytes", "dit_ctx_create", "dit_ctx_destroy", "dit_load_block_weights", "dit_load_parallel_block_weights", "dit_load_dual_block_weights",
            "dit_pack_requests", "dit_pack_tokens", "dit_step_forward", "dit_step_forward_requests", "dit_step_forward_host", "dit_step_forward_host_async", "dit_host_wait",
-           "dit_ctx_poll_status", "dit_debug_tap", "dit_debug_poison", "dit_debug_check_guards", "dit_debug_expire_wait", "dit_debug_attention_probe", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
+           "dit_ctx_poll_status", "dit_debug_tap", "dit_debug_poison", "dit_debug_check_guards", "dit_debug_expire_wait", "dit_debug_clock_probe", "dit_ctx_set_timing", "dit_ctx_read_timing", "dit_modulation_noalloc",
            "dit_load_shell_weights", "dit_timestep_cond", "dit_embed_latents", "dit_final_layer", "dit_sampler_update",
            "dit_denoise_step", "dit_denoise_round", "dit_last_launch_count", "dit_status_string", "dit_last_error"]
 
@@ -125,8 +125,8 @@ def load_library() -> C.CDLL:
     lib.dit_debug_check_guards.argtypes = [vp, C.POINTER(i32)]
     lib.dit_debug_expire_wait.restype = C.c_int
     lib.dit_debug_expire_wait.argtypes = [vp, vp]
-    lib.dit_debug_attention_probe.restype = C.c_int
-    lib.dit_debug_attention_probe.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32)]
+    lib.dit_debug_clock_probe.restype = C.c_int
+    lib.dit_debug_clock_probe.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     lib.dit_ctx_set_timing.restype = C.c_int
     lib.dit_ctx_set_timing.argtypes = [vp, i32]
     lib.dit_ctx_read_timing.restype = C.c_int
@@ -515,11 +515,12 @@ class DitContext:
         """Launches the one-CTA kernel whose bounded wait runs out (sets the status word)."""
         self._check(self.lib.dit_debug_expire_wait(self.handle, self._stream(stream)))
 
-    def dit_debug_attention_probe(self, enabled: bool):
-        """Sets the probe's state; returns (SM MHz inside an attention CTA, cycles per key block) left since the last call."""
-        mhz, cyc = C.c_int32(0), C.c_int32(0)
-        self._check(self.lib.dit_debug_attention_probe(self.handle, 1 if enabled else 0, C.byref(mhz), C.byref(cyc)))
-        return int(mhz.value), int(cyc.value)
+    def dit_debug_clock_probe(self, enabled: bool):
+        """Sets the probe's state; returns (SM MHz inside an attention CTA, its cycles per key block, SM MHz inside a
+        GEMM CTA) left since the last call."""
+        mhz, cyc, gmhz = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+        self._check(self.lib.dit_debug_clock_probe(self.handle, 1 if enabled else 0, C.byref(mhz), C.byref(cyc), C.byref(gmhz)))
+        return int(mhz.value), int(cyc.value), int(gmhz.value)
 
     def dit_ctx_set_timing(self, enabled: bool):
         self._check(self.lib.dit_ctx_set_timing(self.handle, 1 if enabled else 0))

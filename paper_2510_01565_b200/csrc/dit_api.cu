@@ -285,6 +285,7 @@ cudaError_t launch_gemm(const dit_ctx* ctx, const CUtensorMap& tmA, const CUtens
   const int tiles = ((p.M + 2 * gemm_cfg::BM - 1) / (2 * gemm_cfg::BM)) * ((p.N + gemm_cfg::BN - 1) / gemm_cfg::BN);
   const int grid = 2 * std::min(tiles, ctx->gemm_pairs);   // a two-stream launch may have more items than row tiles: the loop covers them
   q.operand_bf16 = (ctx->cfg.flags & DIT_FLAG_BF16_OPERANDS) ? 1 : 0;
+  q.probe = (ctx->attn_probe && p.status) ? p.status + 6 : nullptr;
   gemm_tcgen05_kernel<EPI, HD, DUAL, FP8, BF16><<<grid, gemm_cfg::THREADS, gemm_cfg::SMEM_BYTES, st>>>(tmA, tmB, tmB2 ? *tmB2 : tmB, q, seq, geo);
   return cudaGetLastError();
 }
@@ -1279,15 +1280,17 @@ dit_status dit_debug_check_guards(dit_ctx* ctx, int32_t* n_damaged) {
   return DIT_OK;
 }
 
-dit_status dit_debug_attention_probe(dit_ctx* ctx, int32_t enabled, int32_t* sm_mhz, int32_t* cycles_per_key_block) {
+dit_status dit_debug_clock_probe(dit_ctx* ctx, int32_t enabled, int32_t* attention_mhz, int32_t* cycles_per_key_block,
+                                 int32_t* gemm_mhz) {
   if (!ctx) return DIT_ERR_INVALID_ARG;
   ctx->err[0] = 0;
   DIT_CUDA_TRY(ctx, cudaDeviceSynchronize());
-  int word[2] = {0, 0};
+  int word[3] = {0, 0, 0};
   DIT_CUDA_TRY(ctx, cudaMemcpy(word, ctx->at<int>(ctx->lay.status) + 4, sizeof(word), cudaMemcpyDeviceToHost));
   DIT_CUDA_TRY(ctx, cudaMemset(ctx->at<int>(ctx->lay.status) + 4, 0, sizeof(word)));
-  if (sm_mhz) *sm_mhz = word[0];
+  if (attention_mhz) *attention_mhz = word[0];
   if (cycles_per_key_block) *cycles_per_key_block = word[1];
+  if (gemm_mhz) *gemm_mhz = word[2];
   ctx->attn_probe = enabled != 0;
   return DIT_OK;
 }

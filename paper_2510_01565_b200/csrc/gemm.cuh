@@ -59,6 +59,8 @@ struct GemmParams {
   const float* row_scale;   // [M]
   const float* col_scale;   // [N]
   int operand_bf16;         // A and Wt hold bf16 instead of fp16 (same tensor maps: 16-bit elements)
+  int* probe;               // measurement hook, NULL normally: [0] SM clock in MHz seen by a CTA of this launch
+                            // (cycle counter against the global nanosecond timer over the CTA's life)
 };
 
 namespace gemm_cfg {
@@ -142,6 +144,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   float* epi_stage = reinterpret_cast<float*>(aligned + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  long long probe_c0 = 0; uint64_t probe_t0 = 0;
+  if (p.probe && threadIdx.x == 0) { probe_c0 = clock64(); probe_t0 = global_ns(); }
   const uint32_t rank = cluster_ctarank();                    // 0 = leader of the pair
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_m = DUAL ? *p.num_items : (p.M + 2 * BM - 1) / (2 * BM);   // row tiles (DUAL: row-tile items)
@@ -484,6 +488,11 @@ done:
   cluster_sync_all();        // the peer may still signal this CTA's barriers or read its operands until here
   if (warp == 1) { tc_fence_after(); tmem_dealloc_pair(tmem_base, 512); }
   if (threadIdx.x == 0 && *abort_flag) atomicMax(p.status, kStatusGemmTimeout);
+  if (p.probe && threadIdx.x == 0) {
+    const long long dc = clock64() - probe_c0;
+    const uint64_t dt = global_ns() - probe_t0;
+    if (dt > 20000) p.probe[0] = static_cast<int>(dc * 1000 / static_cast<long long>(dt));   // CTAs that lived 20 us or more
+  }
 }
 
 }  // namespace dit

@@ -440,17 +440,17 @@ def test_bounded_wait_expiry_sets_the_status_word_once(B):
     run.close()
 
 
-def test_attention_probe_reports_a_plausible_clock(B):
+def test_clock_probe_reports_plausible_clocks(B):
     """The measurement hook: attention CTAs of a 1024^2 request (36 key blocks) leave the SM clock they ran at and
-    their cycles per key block; with the hook off nothing is written."""
+    their cycles per key block, GEMM CTAs theirs; with the hook off nothing is written."""
     wl = W.make_custom("probe", W.LARGE, 1, [(1024, 1024, 512)], seed=16)
     run = DeviceRun(B, wl)
-    assert run.ctx.dit_debug_attention_probe(True) == (0, 0)
+    assert run.ctx.dit_debug_clock_probe(True) == (0, 0, 0)
     run.packed()
-    mhz, cyc = run.ctx.dit_debug_attention_probe(False)
-    assert 500 <= mhz <= 2100 and 1500 <= cyc <= 8000, (mhz, cyc)
+    mhz, cyc, gemm_mhz = run.ctx.dit_debug_clock_probe(False)
+    assert 500 <= mhz <= 2100 and 1500 <= cyc <= 8000 and 500 <= gemm_mhz <= 2100, (mhz, cyc, gemm_mhz)
     run.packed()
-    assert run.ctx.dit_debug_attention_probe(False) == (0, 0)
+    assert run.ctx.dit_debug_clock_probe(False) == (0, 0, 0)
     run.close()
 
 
