@@ -292,6 +292,21 @@ def test_widest_hidden_size(B):
     run.close()
 
 
+@pytest.mark.parametrize("hidden,heads,head_dim,mlp,cond", [(64, 1, 64, 64, 1), (128, 1, 128, 64, 3), (192, 3, 64, 320, 5)])
+def test_smallest_dimensions(B, hidden, heads, head_dim, mlp, cond):
+    # the smallest shapes the library accepts: every GEMM is narrower than one 256-column tile and has one or a few
+    # K steps, a single head, a cond vector of one to five channels
+    dims = W.ModelDims(hidden=hidden, n_heads=heads, head_dim=head_dim, mlp_hidden=mlp, cond_dim=cond)
+    wl = W.make_custom("tiny", dims, 2, [(32, 48, 3), (16, 16, 0), (160, 160, 31)], seed=17, timestep_cond=False)
+    run = DeviceRun(B, wl)
+    out = run.packed()
+    ref = oracle_requests(wl, range(3))
+    for r in range(3):
+        check_request(run, out, r, ref[r])
+    check_packed_equals_alone(run, out)
+    run.close()
+
+
 def test_zero_gate_returns_input_exactly(B):
     wl = W.make_custom("zerogate", W.SMALL, 2, [(256, 256, 5), (64, 64, 0)], seed=6, timestep_cond=False)
     H = wl.dims.hidden
