@@ -35,11 +35,11 @@ def f64w(w):
 
 
 class ShellRun:
-    def __init__(self, B, si: W.StepInputs, n_blocks):
+    def __init__(self, B, si: W.StepInputs, n_blocks, flags=0):
         import torch
         self.torch, self.B, self.si, self.nb = torch, B, si, n_blocks
         total = sum(si.token_lens)
-        self.ctx = B.context_for(si.dims, max(n_blocks, 1), total, max(len(si.requests), 1))
+        self.ctx = B.context_for(si.dims, max(n_blocks, 1), total, max(len(si.requests), 1), flags=flags)
         if n_blocks:
             B.upload_weights(self.ctx, si.weights[:n_blocks])
         B.upload_shell_weights(self.ctx, si.shell)
@@ -156,7 +156,7 @@ def _oracle_step(si, n_blocks, latents=None):
                           f64w(si.shell), [f64w(w) for w in si.weights[:n_blocks]], si.dims.n_heads, si.dims.ln_eps)
 
 
-def check_step(run, si, n_blocks):
+def check_step(run, si, n_blocks, tol=TOL):
     torch = run.torch
     before = run.latents.clone()
     vel = torch.empty_like(run.latents)
@@ -166,11 +166,11 @@ def check_step(run, si, n_blocks):
     new, vels, _ = _oracle_step(si, n_blocks)
     for r in range(len(si.requests)):
         err = O.error_metric(run.latent_of(vel, r), vels[r])
-        assert err <= TOL, f"velocity of request {r}: {err:.3e}"
+        assert err <= tol, f"velocity of request {r}: {err:.3e}"
         dz_got = run.latent_of(run.latents, r) - run.latent_of(before, r)
         dz_want = new[r] - si.latents[r].astype(np.float64)
         err = O.error_metric(dz_got, dz_want)
-        assert err <= TOL, f"latent update of request {r}: {err:.3e}"
+        assert err <= tol, f"latent update of request {r}: {err:.3e}"
     return before, vel
 
 
@@ -197,6 +197,19 @@ def test_denoise_step_large_dims_with_text(B):
     si = W.make_step_inputs(W.LARGE, 2, [(256, 256, 64), (512, 256, 0)], seed=16)
     run = ShellRun(B, si, 2)
     check_step(run, si, 2)
+    run.close()
+
+
+def test_denoise_step_with_bf16_operands(B):
+    # the whole step in the bf16-operand mode: the final layer's LayerNorm output and output projection take the
+    # mode's formats too; bar of the mode (6e-2), and the velocity differs from the fp16-operand step's
+    si = W.make_step_inputs(W.SMALL, 2, MIXED_SMALL, seed=19)
+    run16 = ShellRun(B, si, 2)
+    _, vel16 = check_step(run16, si, 2)
+    run16.close()
+    run = ShellRun(B, si, 2, flags=B.DIT_FLAG_BF16_OPERANDS)
+    _, vel = check_step(run, si, 2, tol=6e-2)
+    assert not run.torch.equal(vel, vel16)
     run.close()
 
 
