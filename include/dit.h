@@ -23,7 +23,9 @@
  *   - The caller owns every buffer, including the workspace; the context owns only what it carves
  *     from the workspace.  No entry point below allocates device memory.
  *   - A context is not thread-safe; calls on one context must be issued serially (they may be
- *     asynchronous on one stream).
+ *     asynchronous on one stream).  Different contexts share nothing (the library keeps no state
+ *     outside a context and its workspace, dit_modulation_noalloc's fixed scratch apart) and may
+ *     step at the same time on different streams.
  *
  * The block (per request r, tokens x [L_r, H], cond c [C]); the paper runs such blocks through
  * PyTorch and does not restate them, so this is the standard adaLN-Zero form:
