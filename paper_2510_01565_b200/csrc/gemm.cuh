@@ -9,9 +9,14 @@
 // one CTA per 128x256 tile this halves the shared-memory and L2 traffic for the weight operand.
 // No TMA multicast is used: both CTAs' loads report their bytes to the leader's barrier, and
 // tcgen05.commit (multicast over the pair) releases stages and publishes accumulators in both CTAs.
-// Warp roles: 0 = TMA producer, 1 = MMA issuer (leader CTA only) and TMEM owner, 2..5 = epilogue (one
-// TMEM lane quarter each).  Tiles are taken in a fixed order and every output element is accumulated
-// over K in the same order whatever M is: a row's result does not depend on where it sits in the batch.
+// Warp roles (12 warps = 3 warpgroups): 0 = TMA producer, 1 = MMA issuer (leader CTA only) and TMEM owner,
+// 2..3 = none (they fill the first warpgroup, so that registers can be re-balanced per warpgroup), 4..11 =
+// epilogue: two warps per TMEM lane quarter, one for each half of the tile's columns.  In the steady state the
+// epilogue is hidden under the next tile's main loop; it is exposed in a launch's last wave, which is the whole
+// launch for a small batch, and there eight warps with their requests issued ahead (residual rows before the
+// accumulator is complete, bias / gate / scale vectors one chunk ahead) finish it in half the time of four.
+// Tiles are taken in a fixed order and every output element is accumulated over K in the same order whatever
+// M is: a row's result does not depend on where it sits in the batch.
 //
 // Epilogues (the fused parts of the adaLN-Zero block):
 //   kEpiBiasF16      out16 = acc + bias                                   (QKV projection)
@@ -68,9 +73,16 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 6;     // BM: rows per CTA; 
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = (BN / 2) * BK * 2;                  // this CTA's half of the weight tile
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int THREADS = 192;
-constexpr int EPI_STAGE_FLOATS = 32 * 36;          // per epilogue warp: 32 rows x 32 columns, rows padded to 144 bytes
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * EPI_STAGE_FLOATS * 4;
+constexpr int EPI_WARPS = 8;                       // two per quarter of the accumulator's rows, each takes half of the columns
+// Warpgroup 0 = {TMA warp, MMA warp, two warps without a role}, warpgroups 1 and 2 = epilogue.  Registers are
+// re-balanced per warpgroup (setmaxnreg): each scheduler of the SM hosts one warp of each warpgroup, and ten warps
+// at one common budget would leave the epilogue 168 registers, too few for its residual rows in flight.
+constexpr int THREADS = 128 + 32 * EPI_WARPS;
+constexpr int REGS_ISSUE = 56, REGS_EPILOGUE = 224;   // (56 + 2 * 224) * 32 <= 16384 per scheduler
+// per epilogue warp: 16 rows x 32 fp32 columns with rows padded to 144 bytes (the fp32 epilogues pass their 32 rows
+// through in two halves), or 32 rows x 32 16-bit columns with rows padded to 80 bytes
+constexpr int EPI_STAGE_FLOATS = 640;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_WARPS * EPI_STAGE_FLOATS * 4;
 }  // namespace gemm_cfg
 
 __device__ __forceinline__ float gelu_tanh_f32(float z) {
@@ -161,7 +173,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * EPI_WARPS); }
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -173,6 +185,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  if (warp < 4) {
+    DIT_SETMAXNREG_DEC(REGS_ISSUE);
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
@@ -222,9 +236,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         umma_commit_pair(tfull_bar(acc), 3);       // accumulator complete in both CTAs
       }
     }
+  }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps)
+    DIT_SETMAXNREG_INC(REGS_EPILOGUE);
+    // ------------------------------------------------------------------ epilogue (8 warps)
+    // Two warps share each quarter of the accumulator's rows; the first takes the tile's columns 0..127, the
+    // second 128..255.  When a launch is a single wave (small batches), or in every launch's last wave, the
+    // epilogue is not hidden under a next main loop: twice the warps keep twice the memory requests in flight.
     const int quarter = warp & 3;              // TMEM lanes this warp may read: [32*quarter, +32)
+    const int chalf = (warp - 4) >> 2;         // which half of the tile's columns
+    constexpr int kChunks = BN / 32 / 2;       // 32-column chunks per warp
     int it = 0;
     const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0), tempty_leader1 = map_to_cta(tempty_bar(1), 0);
     for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
@@ -260,10 +281,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (m0 + quarter * 32 + rr < p.M && (!DUAL || rk == kind)) store_rows |= 1u << i8;
         }
       }
-      // Residual rows of this tile do not depend on the accumulator: the first four 32-column chunks
-      // are requested before waiting for the MMAs, later chunks four iterations ahead.
+      // Residual rows of this tile do not depend on the accumulator: three of this warp's four 32-column
+      // chunks are requested before waiting for the MMAs, the fourth when the first has been consumed
+      // (four at once would not fit the register file beside the accumulator chunk).
       const int cg = (lane & 7) * 4;
-      constexpr int kResDepth = 4;             // 32-column chunks of residual rows in flight per lane
+      constexpr int kResDepth = 3;
       float4 xres[kResDepth][8];
       auto load_resid = [&](int c, float4 (&x)[8]) {
         const int col = n0 + c * 32 + cg;
@@ -276,7 +298,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       };
 #pragma unroll
-      for (int d = 0; d < kResDepth; ++d) load_resid(d, xres[d]);
+      for (int d = 0; d < kResDepth; ++d) load_resid(chalf * kChunks + d, xres[d]);
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) goto done;
       tc_fence_after();
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
@@ -289,7 +311,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (local < geo.img_cu[rq + 1] - geo.img_cu[rq]) { py = local / geo.gw[rq]; px = local - py * geo.gw[rq]; }
         }
 #pragma unroll 1
-        for (int hc = 0; hc < BN / HD; ++hc) {
+        for (int hl = 0; hl < BN / HD / 2; ++hl) {
+          const int hc = chalf * (BN / HD / 2) + hl;
           const int colh = n0 + hc * HD;       // first column of this head; heads never straddle Q | K | V
           if (colh >= p.N) break;              // warp-uniform
           float v[HD];
@@ -365,9 +388,39 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       } else {
+      // fp32 epilogues: the bias, gate and column-scale values of a chunk are requested one chunk ahead, so
+      // that their latency passes under the previous chunk's work instead of in front of every chunk
+      float4 nb4 = make_float4(0.f, 0.f, 0.f, 0.f), ng4 = nb4, ncs4 = make_float4(1.f, 1.f, 1.f, 1.f);
+      auto load_vectors = [&](int c) {
+        const int col = n0 + c * 32 + cg;
+        if ((EPI == kEpiGateResidF32 || EPI == kEpiBiasF32) && c < BN / 32 && col < p.N) {
+          nb4 = __ldg(reinterpret_cast<const float4*>(bias + col));
+          if (FP8) ncs4 = __ldg(reinterpret_cast<const float4*>(p.col_scale + col));
+          if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) ng4 = __ldg(reinterpret_cast<const float4*>(gate + req0 * p.gate_stride + col));
+        }
+      };
+      // 16-bit epilogues: the 32 bias values of the next chunk, the same way
+      float4 nbias[8];
+      auto load_bias16 = [&](int c) {
+        const int col0 = n0 + c * 32;
+        if ((EPI == kEpiBiasF16 || EPI == kEpiBiasGeluF16) && c < BN / 32 && col0 + 32 <= p.N) {
 #pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
+          for (int v = 0; v < 8; ++v) nbias[v] = __ldg(reinterpret_cast<const float4*>(bias + col0) + v);
+        }
+      };
+      load_vectors(chalf * kChunks);
+      load_bias16(chalf * kChunks);
+#pragma unroll
+      for (int cl = 0; cl < kChunks; ++cl) {
+        const int c = chalf * kChunks + cl;
         uint32_t r[32];
+        const float4 b = nb4, g_one = ng4, cs = ncs4;
+        float4 bias_now[8];
+        if (EPI == kEpiBiasF16 || EPI == kEpiBiasGeluF16) {
+#pragma unroll
+          for (int v = 0; v < 8; ++v) bias_now[v] = nbias[v];
+        }
+        if (cl + 1 < kChunks) { load_vectors(c + 1); load_bias16(c + 1); }
         __syncwarp();                          // tcgen05.ld is warp-collective: reconverge first
         tmem_ld32(t_row + c * 32, r);
         tmem_ld_wait();
@@ -377,31 +430,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           // Transpose through shared memory so that each global access covers whole 128-byte row
           // segments: lane -> (row it*4 + lane/8, columns (lane%8)*4 .. +3).
           // Rows are padded to 36 floats: 16-byte accesses of both phases are free of bank conflicts.
-          float* st = epi_stage + (warp - 2) * EPI_STAGE_FLOATS;
-#pragma unroll
-          for (int i = 0; i < 32; i += 4)
-            *reinterpret_cast<uint4*>(st + lane * 36 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-          __syncwarp();
+          float* st = epi_stage + (warp - 4) * EPI_STAGE_FLOATS;
           const int col = col0 + cg;                        // N is a multiple of 64: the whole chunk is inside
-          {
-            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + col));
-            float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (FP8) cs = __ldg(reinterpret_cast<const float4*>(p.col_scale + col));
-            float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (EPI == kEpiGateResidF32 && one_req && req0 >= 0) g = __ldg(reinterpret_cast<const float4*>(gate + req0 * p.gate_stride + col));
-            float4 x[8];
-            if (EPI == kEpiGateResidF32) {
+          float4 g = g_one;
 #pragma unroll
-              for (int it = 0; it < 8; ++it) x[it] = xres[c % kResDepth][it];
-              if (c + kResDepth < BN / 32) load_resid(c + kResDepth, xres[c % kResDepth]);
+          for (int hf = 0; hf < 2; ++hf) {                  // rows 0..15 of the warp's 32, then rows 16..31
+            if ((lane >> 4) == hf) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<uint4*>(st + (lane & 15) * 36 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
             }
+            __syncwarp();
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
+            for (int it = hf * 4; it < hf * 4 + 4; ++it) {
               const int rr = it * 4 + (lane >> 3);
               const int grow = m0 + quarter * 32 + rr;
               if ((store_rows >> it) & 1u) {
                 if (EPI == kEpiGateResidF32 && !one_req) g = __ldg(reinterpret_cast<const float4*>(gate + row_req[it] * p.gate_stride + col));
-                const float4 a = *reinterpret_cast<const float4*>(st + rr * 36 + cg);
+                const float4 a = *reinterpret_cast<const float4*>(st + (rr & 15) * 36 + cg);
                 float2 s0, s1;
                 if (FP8) {     // codes back to values: row scale of the activations, column scale of the weights
                   const float sr = row_sa[it];
@@ -413,8 +459,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
                 float4 o;
                 if (EPI == kEpiGateResidF32) {
-                  const float2 o0 = ffma2(make_float2(g.x, g.y), s0, make_float2(x[it].x, x[it].y));
-                  const float2 o1 = ffma2(make_float2(g.z, g.w), s1, make_float2(x[it].z, x[it].w));
+                  const float4 x = xres[cl % kResDepth][it];
+                  const float2 o0 = ffma2(make_float2(g.x, g.y), s0, make_float2(x.x, x.y));
+                  const float2 o1 = ffma2(make_float2(g.z, g.w), s1, make_float2(x.z, x.w));
                   o = make_float4(o0.x, o0.y, o1.x, o1.y);
                 } else {
                   o = make_float4(s0.x, s0.y, s1.x, s1.y);
@@ -422,21 +469,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 *reinterpret_cast<float4*>(p.out32 + static_cast<size_t>(grow) * p.N + col) = o;
               }
             }
+            __syncwarp();                      // the staging buffer is reused by the next half and the next chunk
           }
-          __syncwarp();                        // staging buffer is reused by the next chunk
+          if (EPI == kEpiGateResidF32 && cl + kResDepth < kChunks) load_resid(c + kResDepth, xres[cl % kResDepth]);
         } else {
           const bool full = (col0 + 32 <= p.N);            // warp-uniform
           const int ld = p.ld16 ? p.ld16 : p.N;
           if (full) {
             // fp16 results go through shared memory so that a store instruction covers 64 contiguous
             // bytes of each of 8 rows (whole sectors) instead of 16 bytes of each of 32 rows
-            uint8_t* stb = reinterpret_cast<uint8_t*>(epi_stage + (warp - 2) * EPI_STAGE_FLOATS);
+            uint8_t* stb = reinterpret_cast<uint8_t*>(epi_stage + (warp - 4) * EPI_STAGE_FLOATS);
             uint4* srow = reinterpret_cast<uint4*>(stb + lane * 80);
-            const float4* bias4 = reinterpret_cast<const float4*>(bias + col0);   // col0 is a multiple of 32
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
               uint32_t w[4];
-              const float4 b0 = __ldg(bias4 + 2 * v), b1 = __ldg(bias4 + 2 * v + 1);
+              const float4 b0 = bias_now[2 * v], b1 = bias_now[2 * v + 1];   // col0 is a multiple of 32
               const float2 bb[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
@@ -478,7 +525,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster_light(acc ? tempty_leader1 : tempty_leader0);   // 8 arrivals: 4 warps x 2 CTAs
+      if (lane == 0) mbar_arrive_cluster_light(acc ? tempty_leader1 : tempty_leader0);   // 16 arrivals: 8 warps x 2 CTAs
     }
   }
 
