@@ -21,7 +21,8 @@
 // P V + Q K^T round trip.  TMEM: S 128 columns, P[0], P[1] 64 each, O[0], O[1] 128 each = 512.
 // O is rescaled in TMEM only when a row maximum has grown by more than 2^8 since the reference was
 // set (rare after the first tiles); P is bounded by 2^8, and O and l share the reference, so the
-// normalised result is the same.  Output = acc / l, written as fp16 [T, H].
+// normalised result is the same.  Output = acc / l, written as fp16 [T, H]; a warp passes its 32 rows through
+// the shared memory of the tile's (by then unused) Q so that its stores cover whole rows.
 //
 // Thread layout (384): warpgroup 0 = {warp 0: TMA producer, warp 1: score MMAs + TMEM owner, warp 2: P V MMAs},
 // warpgroups 1 and 2 = softmax for query tile 0 and 1.  Registers are re-balanced with setmaxnreg.
@@ -211,7 +212,6 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
     DIT_SETMAXNREG_INC(200);
     const int tile = (warp >> 2) - 1;                            // query tile of this warpgroup
     const int quarter = warp & 3;
-    const int prow = quarter * 32 + lane;                        // query row inside the tile
     if (len == 0 || (tile == 1 && !tile1_valid)) goto done;
     const uint32_t lane_sel = static_cast<uint32_t>(quarter * 32) << 16;
     const uint32_t tSi = tS + lane_sel, tPi = tP + tile * 64 + lane_sel, tOi = tO + tile * 128 + lane_sel;
@@ -310,27 +310,45 @@ attention_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttnPa
       // reference exactly and a row's probabilities can all underflow or overflow: such a row is written
       // as zeros, never as NaN or infinity
       const float inv = l > 0.f ? 1.0f / l : 0.f;
-      const int row_in_req = qb * C::Q_ROWS + tile * 128 + prow;
-      __half* dst = p.out + static_cast<size_t>(row_begin + row_in_req) * p.ld_out + head * D;
+      // The rows go out through shared memory, so that a store instruction covers 256 contiguous bytes of
+      // each of two rows instead of 16 bytes of each of 32 rows.  The staging area is this tile's Q (all
+      // score products that read it finished before the last P V did); each warp stages its own 32 rows,
+      // 16-byte units XOR-swizzled by the row so that both phases are free of bank conflicts.
+      constexpr int ROW_BYTES = D * 2, UNITS = ROW_BYTES / 16;       // 256 bytes = 16 units for d = 128
+      uint8_t* stage = smem_raw + (((smem_u32(smem_raw) + 1023u) & ~1023u) - smem_u32(smem_raw)) + C::OFF_Q + tile * C::TILE_BYTES + quarter * 32 * ROW_BYTES;
 #pragma unroll 1
       for (int ch = 0; ch < D / 32; ++ch) {
         uint32_t r[32];
         __syncwarp();
         tmem_ld32(tOi + ch * 32, r);
         tmem_ld_wait();
-        if (row_in_req < len) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint32_t w[4];
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              const int i = 8 * v + 2 * h;
-              float o0 = __uint_as_float(r[i]) * inv, o1 = __uint_as_float(r[i + 1]) * inv;
-              if (!(fabsf(o0) <= 3.0e38f)) o0 = 0.f;
-              if (!(fabsf(o1) <= 3.0e38f)) o1 = 0.f;
-              w[h] = pack16x2<BF16>(o0, o1);
-            }
-            *(reinterpret_cast<uint4*>(dst + ch * 32) + v) = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int h = 0; h < 4; ++h) {
+            const int i = 8 * v + 2 * h;
+            float o0 = __uint_as_float(r[i]) * inv, o1 = __uint_as_float(r[i + 1]) * inv;
+            if (!(fabsf(o0) <= 3.0e38f)) o0 = 0.f;
+            if (!(fabsf(o1) <= 3.0e38f)) o1 = 0.f;
+            w[h] = pack16x2<BF16>(o0, o1);
+          }
+          const int unit = ch * 4 + v;
+          *reinterpret_cast<uint4*>(stage + lane * ROW_BYTES + ((unit ^ (lane & (UNITS - 1))) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      __syncwarp();
+      {
+        constexpr int ROWS_PER_STORE = 32 / UNITS;                   // 2 rows per instruction for d = 128, 4 for d = 64
+        const int unit = lane % UNITS, sub = lane / UNITS;
+        const int row0_in_req = qb * C::Q_ROWS + tile * 128 + quarter * 32;
+        __half* out0 = p.out + static_cast<size_t>(row_begin + row0_in_req) * p.ld_out + head * D;
+#pragma unroll 4
+        for (int it = 0; it < 32 / ROWS_PER_STORE; ++it) {
+          const int rr = it * ROWS_PER_STORE + sub;
+          if (row0_in_req + rr < len) {
+            const uint4 val = *reinterpret_cast<const uint4*>(stage + rr * ROW_BYTES + ((unit ^ (rr & (UNITS - 1))) << 4));
+            *(reinterpret_cast<uint4*>(out0 + static_cast<size_t>(rr) * p.ld_out) + unit) = val;
           }
         }
       }
