@@ -39,8 +39,8 @@ DEFAULT_WORKLOAD = "cfg5_mixed8"
 # keys and values (attention) once per band of rows that fits L2, so traffic grows with T and other workloads
 # of the same model are scaled by T / 9216; `traffic_scaled_from` in the JSON line says so.
 NCU_CAPTURE_TOKENS = 9216
-NCU_GEMM_TRAFFIC_BYTES = 503.0e6
-NCU_ATTENTION_TRAFFIC_BYTES = 204.0e6
+NCU_GEMM_TRAFFIC_BYTES = 509.0e6
+NCU_ATTENTION_TRAFFIC_BYTES = 205.0e6
 
 
 def ncu_traffic(wl, bytes_at_capture):
